@@ -1,0 +1,265 @@
+/*
+ * CPU oracle for one segmented-gossip synchronization round
+ * ("Decentralized Federated Learning: A Segmented Gossip Approach", Section 3
+ * and Section 4.1).
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is a plain, slow, single-threaded
+ * statement of what the round computes, used only to check the CUDA library
+ * and to time a CPU baseline.  It shares no code, header, table or constant
+ * generator with the CUDA path and the product never calls it.
+ *
+ * Notation (the paper's): n = N workers, W = flat parameter vector of P
+ * entries, S segments, R model replicas, |D_j| = dataset size of worker j,
+ * P_l = set of workers providing segment l (the worker itself included).
+ *
+ * What is pinned by the CPU tests, function by function:
+ *   oracle_segment_bounds        closed form + partition property
+ *   oracle_splitmix64_next       published splitmix64 output sequence
+ *   oracle_rand32                avalanche / range statistics only
+ *   oracle_select_peers          invariants Section 4.1 step (2) fixes (never
+ *                                self, no repeat, even spread, all distinct
+ *                                when S*R <= n-1), uniformity of the shuffle.
+ *                                Its exact tables are PARITY UNPINNED by the
+ *                                paper, which names no generator.
+ *   oracle_segment_aggregate_*   exact rational brute force of Eq. 3 on tiny
+ *                                inputs, hand-worked dyadic example, R = 0,
+ *                                R = n-1 (all-reduce / FedAvg mean), S = 1,
+ *                                convexity, identical inputs
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------ */
+/* Eq. 1: W = (W[1], ..., W[S]), S non-overlapping segments with the   */
+/* same number of parameters.  Reading for P mod S != 0: segment       */
+/* length ceil(P/S), the last segment(s) shorter, possibly empty.      */
+/* ------------------------------------------------------------------ */
+int64_t oracle_segment_length(int64_t P, int S) { return (P + S - 1) / S; }
+
+void oracle_segment_bounds(int64_t P, int S, int64_t *lo, int64_t *hi) {
+    int64_t L = oracle_segment_length(P, S);
+    for (int l = 0; l < S; ++l) {
+        int64_t a = (int64_t)l * L, b = (int64_t)(l + 1) * L;
+        lo[l] = a < P ? a : P;
+        hi[l] = b < P ? b : P;
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Counter-based random numbers.  The paper only says "randomly        */
+/* selected"; the generator below is this library's definition:        */
+/* splitmix64 (Steele, Lea, Flood, OOPSLA 2014) and a keyed chain of   */
+/* its output function over the counter (seed, round|w, epoch|t).      */
+/* ------------------------------------------------------------------ */
+static uint64_t sm64_mix(uint64_t z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+
+/* One step of the splitmix64 generator: advances *state, returns output. */
+uint64_t oracle_splitmix64_next(uint64_t *state) {
+    *state += 0x9E3779B97F4A7C15ULL;
+    return sm64_mix(*state);
+}
+
+/* rand32(seed, round, w, e, t): three chained splitmix64 steps, each
+ * started from the previous output xor the next counter word; the result
+ * is the high half of the last output. */
+uint32_t oracle_rand32(uint64_t seed, uint32_t round, uint32_t w, uint32_t e, uint32_t t) {
+    uint64_t s = seed;
+    uint64_t h = oracle_splitmix64_next(&s);
+    s = h ^ (((uint64_t)round << 32) | (uint64_t)w);
+    h = oracle_splitmix64_next(&s);
+    s = h ^ (((uint64_t)e << 32) | (uint64_t)t);
+    h = oracle_splitmix64_next(&s);
+    return (uint32_t)(h >> 32);
+}
+
+/* ------------------------------------------------------------------ */
+/* Section 4.1 step (2): each worker issues S*R pull requests; every   */
+/* target is drawn at random from all the OTHER workers without        */
+/* replacement until no option is left.  Readings: after the pool is   */
+/* exhausted a fresh random order of the others starts (new epoch);    */
+/* P_l in Eq. 3 is a set, so a segment never gets one peer twice: the  */
+/* peers already chosen for the current segment are moved, in order,   */
+/* behind the rest of a freshly shuffled pool.                         */
+/* idx layout [w][l][r], each (w,l) row ascending.                     */
+/* Returns 0, or 1 for invalid arguments.                              */
+/* ------------------------------------------------------------------ */
+static int cmp_i32(const void *a, const void *b) {
+    int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+int oracle_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t *idx) {
+    if (N < 1 || S < 1 || R < 0 || R > N - 1) return 1;
+    if (R == 0) return 0;
+    int M = N - 1;
+    int32_t *perm = (int32_t *)malloc(sizeof(int32_t) * (size_t)M);
+    int32_t *tmp = (int32_t *)malloc(sizeof(int32_t) * (size_t)M);
+    int32_t *chosen = (int32_t *)malloc(sizeof(int32_t) * (size_t)R);
+    for (int w = 0; w < N; ++w) {
+        int pos = M;          /* pool empty: the first draw opens epoch 0 */
+        uint32_t epoch = 0;
+        int opened = 0;
+        for (int l = 0; l < S; ++l) {
+            int nc = 0;
+            for (int r = 0; r < R; ++r) {
+                if (pos == M) {
+                    if (opened) ++epoch;
+                    opened = 1;
+                    /* all the other workers, ascending */
+                    for (int i = 0, v = 0; v < N; ++v)
+                        if (v != w) perm[i++] = v;
+                    /* Fisher-Yates shuffle, t = M-1 down to 1 */
+                    for (int t = M - 1; t >= 1; --t) {
+                        uint32_t u = oracle_rand32(seed, round, (uint32_t)w, epoch, (uint32_t)t);
+                        int j = (int)(((uint64_t)u * (uint64_t)(t + 1)) >> 32);
+                        int32_t s = perm[t]; perm[t] = perm[j]; perm[j] = s;
+                    }
+                    /* peers this segment already has go to the back, stably */
+                    if (nc > 0) {
+                        int a = 0;
+                        for (int i = 0; i < M; ++i) {
+                            int taken = 0;
+                            for (int c = 0; c < nc; ++c) taken |= (chosen[c] == perm[i]);
+                            if (!taken) tmp[a++] = perm[i];
+                        }
+                        for (int i = 0; i < M; ++i) {
+                            int taken = 0;
+                            for (int c = 0; c < nc; ++c) taken |= (chosen[c] == perm[i]);
+                            if (taken) tmp[a++] = perm[i];
+                        }
+                        memcpy(perm, tmp, sizeof(int32_t) * (size_t)M);
+                    }
+                    pos = 0;
+                }
+                chosen[nc++] = perm[pos++];
+            }
+            qsort(chosen, (size_t)R, sizeof(int32_t), cmp_i32);
+            memcpy(idx + ((size_t)w * S + l) * R, chosen, sizeof(int32_t) * (size_t)R);
+        }
+    }
+    free(perm); free(tmp); free(chosen);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* bf16 <-> binary32/binary64 (bf16 = the upper 16 bits of binary32).  */
+/* ------------------------------------------------------------------ */
+static float bf16_to_f32(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f; memcpy(&f, &u, 4); return f;
+}
+
+/* round-to-nearest-even binary32 -> bf16 (finite inputs) */
+uint16_t oracle_f32_to_bf16_rne(float f) {
+    uint32_t u; memcpy(&u, &f, 4);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 3 and Eq. 4, evaluated as written, in binary64:                 */
+/*   out[w][p] = sum_{j in P_l} |D_j| x_j[p]  /  sum_{j in P_l} |D_j|  */
+/* with l the segment holding p and P_l = {w} U idx[w][l][0..R).       */
+/* x_j[p] is the value worker j SENDS: its locally updated model       */
+/* (Section 4.1 steps 1 and 3), i.e. in[j][p] - lr*grads[j][p] when    */
+/* grads is given, in[j][p] otherwise.                                 */
+/*                                                                     */
+/* `in`/`grads` point at a slab [N][pitch] whose column 0 is global    */
+/* column p_begin; columns [p_begin, p_end) are evaluated and written  */
+/* to out as [N][p_end-p_begin] doubles.  elem = 4: binary32 input,    */
+/* elem = 2: bf16 input.  weights == NULL means |D_j| = 1 for all j.   */
+/* ------------------------------------------------------------------ */
+static double load_x(const void *base, int elem, size_t off) {
+    if (elem == 4) return (double)((const float *)base)[off];
+    return (double)bf16_to_f32(((const uint16_t *)base)[off]);
+}
+
+int oracle_segment_aggregate(const void *in, const void *grads, double lr, int elem,
+                             int64_t pitch, const float *weights, const int32_t *idx,
+                             int N, int64_t P, int S, int R,
+                             int64_t p_begin, int64_t p_end, double *out) {
+    if (N < 1 || P < 1 || S < 1 || R < 0 || R > N - 1) return 1;
+    if (p_begin < 0 || p_end > P || p_begin > p_end) return 1;
+    if (elem != 4 && elem != 2) return 1;
+    int64_t L = oracle_segment_length(P, S);
+    int64_t width = p_end - p_begin;
+    for (int w = 0; w < N; ++w) {
+        for (int64_t p = p_begin; p < p_end; ++p) {
+            int l = (int)(p / L);
+            const int32_t *peers = idx ? idx + ((size_t)w * S + l) * R : NULL;
+            double num = 0.0, den = 0.0;
+            for (int m = -1; m < R; ++m) {
+                int j = (m < 0) ? w : peers[m];
+                size_t off = (size_t)j * (size_t)pitch + (size_t)(p - p_begin);
+                double x = load_x(in, elem, off);
+                if (grads) x = x - lr * load_x(grads, elem, off);
+                double D = weights ? (double)weights[j] : 1.0;
+                num += D * x;
+                den += D;
+            }
+            out[(size_t)w * (size_t)width + (size_t)(p - p_begin)] = num / den;
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* The same round in binary32 with one fixed operation order: provider */
+/* order is self first, then peers ascending; the weights are          */
+/* normalised first (c_j = |D_j| / sum, one IEEE division per          */
+/* provider), then out = c_self*x_self, out = fma(c_j, x_j, out).      */
+/* The local step is x = fma(-lr, g, x) rounded to binary32.  A bf16   */
+/* result is the binary32 result rounded to nearest even.  This is a   */
+/* second, tighter yardstick for a binary32 implementation that uses   */
+/* the same order; it is itself pinned against the binary64 form.      */
+/* out: [N][p_end-p_begin] of float (elem 4) or uint16 bf16 (elem 2).  */
+/* ------------------------------------------------------------------ */
+int oracle_segment_aggregate_ordered_f32(const void *in, const void *grads, float lr, int elem,
+                                         int64_t pitch, const float *weights, const int32_t *idx,
+                                         int N, int64_t P, int S, int R,
+                                         int64_t p_begin, int64_t p_end, void *out) {
+    if (N < 1 || P < 1 || S < 1 || R < 0 || R > N - 1) return 1;
+    if (p_begin < 0 || p_end > P || p_begin > p_end) return 1;
+    if (elem != 4 && elem != 2) return 1;
+    if (grads && elem != 4) return 1;
+    int64_t L = oracle_segment_length(P, S);
+    int64_t width = p_end - p_begin;
+    float *coef = (float *)malloc(sizeof(float) * (size_t)(R + 1));
+    for (int w = 0; w < N; ++w) {
+        for (int l = 0; l < S; ++l) {
+            int64_t a = (int64_t)l * L, b = a + L;
+            if (a < p_begin) a = p_begin;
+            if (b > p_end) b = p_end;
+            if (a >= b) continue;
+            const int32_t *peers = idx ? idx + ((size_t)w * S + l) * R : NULL;
+            volatile float den = weights ? weights[w] : 1.0f;
+            for (int r = 0; r < R; ++r) den = den + (weights ? weights[peers[r]] : 1.0f);
+            coef[0] = (weights ? weights[w] : 1.0f) / den;
+            for (int r = 0; r < R; ++r) coef[r + 1] = (weights ? weights[peers[r]] : 1.0f) / den;
+            for (int64_t p = a; p < b; ++p) {
+                float acc = 0.0f;
+                for (int m = -1; m < R; ++m) {
+                    int j = (m < 0) ? w : peers[m];
+                    size_t off = (size_t)j * (size_t)pitch + (size_t)(p - p_begin);
+                    float x = (elem == 4) ? ((const float *)in)[off]
+                                          : bf16_to_f32(((const uint16_t *)in)[off]);
+                    if (grads) x = fmaf(-lr, ((const float *)grads)[off], x);
+                    if (m < 0) { volatile float prod = coef[0] * x; acc = prod; }
+                    else acc = fmaf(coef[m + 1], x, acc);
+                }
+                size_t o = (size_t)w * (size_t)width + (size_t)(p - p_begin);
+                if (elem == 4) ((float *)out)[o] = acc;
+                else ((uint16_t *)out)[o] = oracle_f32_to_bf16_rne(acc);
+            }
+        }
+    }
+    free(coef);
+    return 0;
+}
