@@ -1,0 +1,194 @@
+/*
+ * combo_b200 -- one synchronization round of segmented gossip aggregation
+ * ("Decentralized Federated Learning: A Segmented Gossip Approach") for N
+ * simulated workers whose flat parameter vectors sit in one GPU's memory.
+ *
+ * C ABI of libcombo_b200.so (CUDA, sm_100a only; there is no CPU or other
+ * fallback).  Plain pointers and sizes; the caller owns every buffer.  Unless
+ * a function says otherwise, pointers are DEVICE pointers of the current
+ * device, calls only enqueue work on the given stream and never synchronise,
+ * and the library allocates nothing.
+ *
+ * Notation follows the paper: n = N workers, S segments, R model replicas,
+ * |D_j| dataset size of worker j, P_l the set of workers providing segment l.
+ *
+ * Layouts
+ *   parameters  [N][P] row-major, worker-major, dense (row pitch = P elements)
+ *   idx         int32 [N][S][R]; idx[w][l][r] = r-th peer of worker w for
+ *               segment l; each (w,l) row ascending, all entries != w, distinct
+ *   weights     float [N], |D_j| > 0, un-normalised; NULL = all equal
+ *
+ * Segments (Eq. 1; the paper's "divided into S segments equally"): segment
+ * length L = ceil(P/S); segment l covers columns [min(l*L,P), min((l+1)*L,P)),
+ * so the last segment is shorter when S does not divide P and trailing
+ * segments may be empty.
+ */
+#ifndef COMBO_B200_H
+#define COMBO_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int combo_status;
+
+enum {
+    COMBO_OK = 0,                 /* work enqueued (or, for host calls, done)    */
+    COMBO_ERR_INVALID_ARG = 1,    /* size out of range, NULL or misaligned pointer */
+    COMBO_ERR_ALIAS = 2,          /* input and output ranges overlap             */
+    COMBO_ERR_UNSUPPORTED = 3,    /* current device is not compute capability 10.x */
+    COMBO_ERR_CUDA = 4,           /* a CUDA runtime call failed; see combo_last_cuda_error */
+    COMBO_ERR_DEVICE_TIMEOUT = 5  /* a bounded wait inside a kernel ran out      */
+};
+
+/* Limits of this build. */
+#define COMBO_MAX_WORKERS 8192    /* N */
+#define COMBO_MAX_SEGMENTS 65536  /* S */
+
+/*
+ * Peer selection -- Section 4.1, step (2) "Segments Pulling": every worker
+ * issues S*R pull requests; each target is drawn at random from all the OTHER
+ * workers, without replacement, until no option is left.  When the pool of
+ * N-1 others is exhausted a freshly shuffled pool is opened; peers already
+ * chosen for the segment being filled are skipped (P_l of Eq. 3 is a set).
+ * Hence: never the worker itself, R distinct peers per (worker, segment), all
+ * S*R peers of a worker distinct when S*R <= N-1, otherwise every other worker
+ * is used floor or ceil of S*R/(N-1) times.
+ *
+ * The table is a pure function of (seed, round, N, S, R): random numbers come
+ * from a counter-based generator (splitmix64 steps chained over the words
+ * seed, round|worker, epoch|position; Fisher-Yates shuffle with the
+ * multiply-shift range reduction), so the call can be issued ahead of the
+ * local update, as the paper notes for the pull requests.
+ *
+ * idx_out: device int32[N*S*R], written completely; not touched when R == 0.
+ * Requires 1 <= N <= COMBO_MAX_WORKERS, 1 <= S <= COMBO_MAX_SEGMENTS,
+ * 0 <= R <= N-1.  combo_select_peers enqueues on the legacy default stream;
+ * the _async form on `stream` (a cudaStream_t passed as void*).
+ */
+combo_status combo_select_peers(uint64_t seed, uint32_t round, int N, int S, int R,
+                                int32_t* idx_out);
+combo_status combo_select_peers_async(uint64_t seed, uint32_t round, int N, int S, int R,
+                                      int32_t* idx_out, void* stream);
+
+/*
+ * Segment-wise aggregation -- Eq. 3 and Eq. 4 (Section 3, "Segmented
+ * Aggregation"), for all N workers at once:
+ *
+ *   out[w][p] = sum_{j in P_l(w)} |D_j| * in[j][p]  /  sum_{j in P_l(w)} |D_j|
+ *
+ * with l the segment that holds column p and P_l(w) = {w} U idx[w][l][0..R).
+ * Every worker reads the same pre-aggregation inputs (workers send the model
+ * they hold after the local update, Section 4.1 steps 3 and 4), so params_out
+ * must not overlap params_in.
+ *
+ * Arithmetic: binary32.  den = |D_w| + |D_k1| + ... (peers ascending),
+ * c_j = |D_j| / den (IEEE division), out = c_w*x_w, then out = fma(c_k, x_k, out)
+ * for the peers in ascending order.  No fast-math, denormals kept.
+ *
+ * params_in, params_out: float [N][P], base addresses 16-byte aligned.
+ * weights: float[N] or NULL.  idx: int32[N][S][R], trusted (see
+ * combo_validate_idx); may be NULL when R == 0.  1 <= P, 0 <= R <= N-1.
+ * R == 0 copies the input bit for bit.
+ */
+combo_status combo_segment_aggregate(const float* params_in, float* params_out,
+                                     const float* weights, const int32_t* idx,
+                                     int N, int64_t P, int S, int R, void* stream);
+
+/*
+ * The same with parameters stored as bfloat16 (uint16_t bit patterns):
+ * inputs are widened exactly, accumulation is binary32 as above, the result
+ * is rounded to nearest even.  Rows need not be 16-byte aligned (odd P*2
+ * pitches are handled); the base addresses must be.
+ */
+combo_status combo_segment_aggregate_bf16(const uint16_t* params_in, uint16_t* params_out,
+                                          const float* weights, const int32_t* idx,
+                                          int N, int64_t P, int S, int R, void* stream);
+
+/*
+ * Local step fused in front of the aggregation -- Section 4.1 step (1) with
+ * one SGD step (tau = 1) on a supplied gradient: every worker j first forms
+ * x'_j = fma(-lr, grads[j], params_in[j]) (binary32), and Eq. 3 is evaluated
+ * on the x'.  Peers contribute their UPDATED rows, exactly as if the step had
+ * been applied to all of params_in before combo_segment_aggregate.  grads:
+ * float [N][P], 16-byte aligned, must not overlap params_out.
+ */
+combo_status combo_segment_aggregate_sgd(const float* params_in, const float* grads, float lr,
+                                         float* params_out, const float* weights,
+                                         const int32_t* idx, int N, int64_t P, int S, int R,
+                                         void* stream);
+
+/*
+ * Column-sharded form of the three calls above, for a vector of P_total
+ * parameters whose columns [p_begin, p_begin + width) are held locally as
+ * [N][pitch] arrays (pitch >= width elements; local column 0 = global column
+ * p_begin).  Eq. 3 couples workers only at equal p, so shards need no
+ * exchange; segment bounds are those of the P_total-vector.
+ * elem_bytes: 4 = float, 2 = bfloat16.  grads may be NULL (no local step;
+ * must be NULL for bfloat16).
+ */
+combo_status combo_segment_aggregate_cols(const void* params_in, const void* grads, float lr,
+                                          void* params_out, int elem_bytes,
+                                          const float* weights, const int32_t* idx,
+                                          int N, int64_t P_total, int S, int R,
+                                          int64_t p_begin, int64_t width, int64_t pitch,
+                                          void* stream);
+
+/*
+ * Checks an idx table on the device: every entry in [0,N), != its worker,
+ * each (w,l) row strictly ascending.  dev_flag: device int32, set to 0 first,
+ * then to 1 + (index of an offending entry) if any check fails.
+ */
+combo_status combo_validate_idx(const int32_t* idx, int N, int S, int R, void* stream,
+                                int32_t* dev_flag);
+
+/*
+ * Whole rounds from HOST memory (the paper's worker iteration, steps 2-4, for
+ * all workers): copies h_params_in (and h_grads, h_weights when given) to the
+ * device buffers, then for t = round .. round+rounds-1 selects peers for
+ * (seed, t) and aggregates, ping-ponging between d_in and d_out, and copies
+ * the final parameters to h_params_out; all on `stream`, which is
+ * synchronised before returning.  With h_grads the fused local step uses the
+ * same gradient array in every round.  Host buffers should be page-locked
+ * for full copy speed.  Device buffers are the caller's: d_in, d_out (and
+ * d_grads if h_grads != NULL) [N][P] of elem_bytes each, d_weights float[N]
+ * (if h_weights != NULL), d_idx int32[N*S*R].  h_idx_out, if not NULL,
+ * receives the peer table of the last round.  rounds >= 1.
+ */
+combo_status combo_round_host(const void* h_params_in, const void* h_grads, float lr,
+                              void* h_params_out, int elem_bytes, const float* h_weights,
+                              uint64_t seed, uint32_t round, int rounds, int N, int64_t P, int S,
+                              int R, void* d_in, void* d_grads, void* d_out, float* d_weights,
+                              int32_t* d_idx, int32_t* h_idx_out, void* stream);
+
+/*
+ * Reads and clears the device status word that kernels set when one of their
+ * bounded waits gives up.  Synchronises the device.  Returns COMBO_OK or
+ * COMBO_ERR_DEVICE_TIMEOUT (or COMBO_ERR_CUDA).
+ */
+combo_status combo_device_status(void);
+
+/* Which aggregation kernel the last combo_segment_aggregate* call on this
+ * thread launched: 0 none, 1 direct gather, 2 shared-memory staged. */
+int combo_last_kernel_path(void);
+
+/* Forces a path for the following calls on this thread: 0 automatic (default),
+ * 1 direct gather, 2 staged (falls back to direct where staging cannot apply). */
+void combo_set_kernel_path(int path);
+
+/* Expert knob for the staged kernel, this thread only: tile width in elements
+ * (a multiple of 128 for float, 256 for bfloat16) and number of pipeline
+ * stages; 0 = chosen automatically.  A tile that cannot be honoured makes
+ * the call fall back to the direct kernel. */
+void combo_set_tuning(int tile_elems, int stages);
+
+const char* combo_status_string(combo_status status);
+const char* combo_last_cuda_error(void);
+int combo_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMBO_B200_H */

@@ -1,0 +1,387 @@
+// libcombo_b200.so: C ABI over the sm_100a kernels (argument checks, tile
+// planning, launches).  See include/combo_b200.h for the contract.
+#include "../../include/combo_b200.h"
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "segment_aggregate.cuh"
+#include "select_peers.cuh"
+
+namespace {
+
+using combo::AggParams;
+
+thread_local char t_cuda_err[256] = "";
+thread_local int t_last_path = 0;
+thread_local int t_force_path = 0;
+thread_local int t_tile = 0;
+thread_local int t_stages = 0;
+
+struct DeviceInfo {
+    int known;       // 0 unknown, 1 supported, -1 unsupported
+    int sms;
+    int smem_optin;
+};
+DeviceInfo g_dev[64];
+
+combo_status cuda_fail(cudaError_t e, const char* what) {
+    snprintf(t_cuda_err, sizeof(t_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+    return COMBO_ERR_CUDA;
+}
+
+combo_status device_info(DeviceInfo** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return COMBO_ERR_UNSUPPORTED;
+    DeviceInfo& d = g_dev[dev];
+    if (d.known == 0) {
+        int major = 0, sms = 0, smem = 0;
+        if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+            return cuda_fail(e, "cudaDeviceGetAttribute");
+        d.sms = sms;
+        d.smem_optin = smem;
+        d.known = (major == 10) ? 1 : -1;
+    }
+    if (d.known < 0) return COMBO_ERR_UNSUPPORTED;
+    *out = &d;
+    return COMBO_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline bool overlaps(const void* a, const void* b, size_t bytes) {
+    uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + bytes && y < x + bytes;
+}
+
+inline unsigned round_up(unsigned v, unsigned q) { return (v + q - 1) / q * q; }
+
+// ---------------------------------------------------------------- staged plan
+struct StagedPlan {
+    bool ok;
+    int gb;          // shared-memory read granule in bytes
+    size_t smem;
+    int grid;
+};
+
+StagedPlan plan_staged(AggParams& p, int EB, bool sgd, const DeviceInfo& dev) {
+    StagedPlan plan = {false, 16, 0, 0};
+    const int V = 16 / EB;
+    const int narr = sgd ? 2 : 1;
+    const bool unaligned = (p.pitch % V) != 0;
+    if (p.R > combo::kStagedMaxR) return plan;
+    p.halo = unaligned ? V : 0;
+    plan.gb = !unaligned ? 16 : (EB == 4 ? 4 : ((p.pitch % 2 == 0) ? 4 : 2));
+    const int Tq = 32 * V;
+    const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
+    const unsigned table = round_up(2u * p.N * ((p.R > 0 ? p.R : 1) * 4u + (p.R + 1) * 4u), 128);
+    const long long budget = (long long)dev.smem_optin - header - table - 128;
+    auto row_bytes = [&](int T) { return (T + p.halo) * EB + (p.halo ? 16 : 0); };
+    auto stage_bytes = [&](int T) { return (long long)round_up((unsigned)(p.N * row_bytes(T) * narr), 128); };
+    auto tiles = [&](int T) { return (p.width + (p.halo ? V - 1 : 0) + T - 1) / T; };
+    if ((long long)Tq + p.halo > p.L) return plan;
+    if (2 * stage_bytes(Tq) > budget) return plan;
+
+    int T = 0;
+    if (t_tile > 0) {
+        if (t_tile % Tq != 0 || (long long)t_tile + p.halo > p.L || 2 * stage_bytes(t_tile) > budget) return plan;
+        T = t_tile;
+    } else {
+        // largest tile whose stage stays near 64 KB, then the candidate with the least
+        // (waves x tile width), a fixed per-tile cost of 32 columns added
+        const long long target = 64 * 1024;
+        int T_hi = Tq;
+        while (T_hi + Tq <= 4096 && (long long)T_hi + Tq + p.halo <= p.L && stage_bytes(T_hi + Tq) <= target &&
+               2 * stage_bytes(T_hi + Tq) <= budget)
+            T_hi += Tq;
+        double best = 0.0;
+        for (int c = T_hi; c >= Tq; c -= Tq) {
+            const long long nt = tiles(c);
+            const long long waves = (nt + dev.sms - 1) / dev.sms;
+            const double cost = (double)waves * (c + 32);
+            if (T == 0 || cost < best * 0.999) { best = cost; T = c; }
+        }
+    }
+    int stages = (int)(budget / stage_bytes(T));
+    if (stages > combo::kMaxStages) stages = combo::kMaxStages;
+    if (t_stages > 0 && t_stages < stages) stages = t_stages;
+    if (stages < 2) return plan;
+    p.T = T;
+    p.stages = stages;
+    p.row_bytes = row_bytes(T);
+    p.stage_bytes = (unsigned)stage_bytes(T);
+    p.tab_off = header;
+    p.stage_off = header + table;
+    p.n_tiles = tiles(T);
+    plan.smem = (size_t)p.stage_off + (size_t)stages * p.stage_bytes;
+    plan.grid = (int)(p.n_tiles < dev.sms ? p.n_tiles : dev.sms);
+    plan.ok = plan.grid > 0;
+    return plan;
+}
+
+template <int EB, int GB, bool SGD, int RT>
+cudaError_t launch_staged_inst(const AggParams& p, const StagedPlan& plan, cudaStream_t st) {
+    auto kern = combo::k_staged<EB, GB, SGD, RT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem);
+    if (e != cudaSuccess) return e;
+    kern<<<plan.grid, combo::kStagedThreads, plan.smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+template <int EB, int GB, bool SGD>
+cudaError_t launch_staged_r(const AggParams& p, const StagedPlan& plan, cudaStream_t st, bool specialise) {
+    if (specialise) {
+        switch (p.R) {
+            case 2: return launch_staged_inst<EB, GB, SGD, 2>(p, plan, st);
+            case 3: return launch_staged_inst<EB, GB, SGD, 3>(p, plan, st);
+            case 4: return launch_staged_inst<EB, GB, SGD, 4>(p, plan, st);
+            default: break;
+        }
+    }
+    return launch_staged_inst<EB, GB, SGD, -1>(p, plan, st);
+}
+
+cudaError_t launch_staged(const AggParams& p, const StagedPlan& plan, int EB, bool sgd, cudaStream_t st) {
+    if (EB == 4) {
+        if (plan.gb == 16) return sgd ? launch_staged_r<4, 16, true>(p, plan, st, true)
+                                      : launch_staged_r<4, 16, false>(p, plan, st, true);
+        return sgd ? launch_staged_r<4, 4, true>(p, plan, st, false) : launch_staged_r<4, 4, false>(p, plan, st, false);
+    }
+    if (plan.gb == 16) return launch_staged_r<2, 16, false>(p, plan, st, true);
+    if (plan.gb == 4) return launch_staged_r<2, 4, false>(p, plan, st, true);
+    return launch_staged_r<2, 2, false>(p, plan, st, false);
+}
+
+cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo& dev, cudaStream_t st) {
+    const int V = 16 / EB;
+    const long long items = ((p.width + V - 1) / V + 1) * (long long)p.N;
+    long long blocks = (items + 255) / 256;
+    const long long cap = (long long)dev.sms * 32;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (EB == 4) {
+        if (sgd) combo::k_direct<4, true><<<(int)blocks, 256, 0, st>>>(p);
+        else combo::k_direct<4, false><<<(int)blocks, 256, 0, st>>>(p);
+    } else {
+        combo::k_direct<2, false><<<(int)blocks, 256, 0, st>>>(p);
+    }
+    return cudaGetLastError();
+}
+
+combo_status aggregate_cols(const void* in, const void* grads, float lr, void* out, int EB,
+                            const float* weights, const int32_t* idx, int N, long long P_total, int S, int R,
+                            long long p_begin, long long width, long long pitch, void* stream) {
+    if (EB != 4 && EB != 2) return COMBO_ERR_INVALID_ARG;
+    if (N < 1 || N > COMBO_MAX_WORKERS || S < 1 || S > COMBO_MAX_SEGMENTS || R < 0 || R > N - 1)
+        return COMBO_ERR_INVALID_ARG;
+    if (P_total < 1 || p_begin < 0 || width < 1 || p_begin + width > P_total || pitch < width)
+        return COMBO_ERR_INVALID_ARG;
+    if (!in || !out || (R > 0 && !idx)) return COMBO_ERR_INVALID_ARG;
+    if (grads && EB != 4) return COMBO_ERR_INVALID_ARG;
+    if (!aligned16(in) || !aligned16(out) || (grads && !aligned16(grads))) return COMBO_ERR_INVALID_ARG;
+    if ((unsigned long long)pitch > (1ull << 40) / (unsigned)N) return COMBO_ERR_INVALID_ARG;
+    const size_t extent = (size_t)(((long long)(N - 1) * pitch + width) * EB);
+    if (overlaps(in, out, extent) || (grads && overlaps(grads, out, extent))) return COMBO_ERR_ALIAS;
+
+    DeviceInfo* dev = nullptr;
+    combo_status rc = device_info(&dev);
+    if (rc != COMBO_OK) return rc;
+
+    AggParams p;
+    memset(&p, 0, sizeof(p));
+    p.in = static_cast<const unsigned char*>(in);
+    p.grads = static_cast<const unsigned char*>(grads);
+    p.out = static_cast<unsigned char*>(out);
+    p.weights = weights;
+    p.idx = idx;
+    p.pitch = pitch;
+    p.p_begin = p_begin;
+    p.width = width;
+    p.L = (P_total + S - 1) / S;
+    p.arr_end_al = (long long)(extent & ~(size_t)15);
+    p.N = N; p.S = S; p.R = R;
+    p.lr = lr;
+    const bool sgd = grads != nullptr;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    bool want_staged = t_force_path != 1;
+    if (t_force_path == 0 && (long long)N * width < (1 << 16)) want_staged = false;   // too small to pipeline
+    if (want_staged) {
+        StagedPlan plan = plan_staged(p, EB, sgd, *dev);
+        if (plan.ok) {
+            cudaError_t e = launch_staged(p, plan, EB, sgd, st);
+            if (e != cudaSuccess) return cuda_fail(e, "staged aggregation launch");
+            t_last_path = 2;
+            return COMBO_OK;
+        }
+    }
+    cudaError_t e = launch_direct(p, EB, sgd, *dev, st);
+    if (e != cudaSuccess) return cuda_fail(e, "direct aggregation launch");
+    t_last_path = 1;
+    return COMBO_OK;
+}
+
+combo_status select_peers_impl(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* idx_out,
+                               cudaStream_t st) {
+    if (N < 1 || N > COMBO_MAX_WORKERS || S < 1 || S > COMBO_MAX_SEGMENTS || R < 0 || R > N - 1)
+        return COMBO_ERR_INVALID_ARG;
+    if (R == 0) return COMBO_OK;
+    if (!idx_out) return COMBO_ERR_INVALID_ARG;
+    DeviceInfo* dev = nullptr;
+    combo_status rc = device_info(&dev);
+    if (rc != COMBO_OK) return rc;
+    const size_t smem = combo::select_peers_smem_bytes(N);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(combo::k_select_peers, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(select_peers)");
+    }
+    combo::k_select_peers<<<N, combo::kSelectThreads, smem, st>>>(seed, round, N, S, R, idx_out);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "select_peers launch");
+    return COMBO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+combo_status combo_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* idx_out) {
+    return select_peers_impl(seed, round, N, S, R, idx_out, (cudaStream_t)0);
+}
+
+combo_status combo_select_peers_async(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* idx_out,
+                                      void* stream) {
+    return select_peers_impl(seed, round, N, S, R, idx_out, static_cast<cudaStream_t>(stream));
+}
+
+combo_status combo_segment_aggregate(const float* params_in, float* params_out, const float* weights,
+                                     const int32_t* idx, int N, int64_t P, int S, int R, void* stream) {
+    return aggregate_cols(params_in, nullptr, 0.0f, params_out, 4, weights, idx, N, P, S, R, 0, P, P, stream);
+}
+
+combo_status combo_segment_aggregate_bf16(const uint16_t* params_in, uint16_t* params_out, const float* weights,
+                                          const int32_t* idx, int N, int64_t P, int S, int R, void* stream) {
+    return aggregate_cols(params_in, nullptr, 0.0f, params_out, 2, weights, idx, N, P, S, R, 0, P, P, stream);
+}
+
+combo_status combo_segment_aggregate_sgd(const float* params_in, const float* grads, float lr, float* params_out,
+                                         const float* weights, const int32_t* idx, int N, int64_t P, int S, int R,
+                                         void* stream) {
+    if (!grads) return COMBO_ERR_INVALID_ARG;
+    return aggregate_cols(params_in, grads, lr, params_out, 4, weights, idx, N, P, S, R, 0, P, P, stream);
+}
+
+combo_status combo_segment_aggregate_cols(const void* params_in, const void* grads, float lr, void* params_out,
+                                          int elem_bytes, const float* weights, const int32_t* idx, int N,
+                                          int64_t P_total, int S, int R, int64_t p_begin, int64_t width,
+                                          int64_t pitch, void* stream) {
+    return aggregate_cols(params_in, grads, lr, params_out, elem_bytes, weights, idx, N, P_total, S, R, p_begin,
+                          width, pitch, stream);
+}
+
+combo_status combo_validate_idx(const int32_t* idx, int N, int S, int R, void* stream, int32_t* dev_flag) {
+    if (N < 1 || S < 1 || R < 0 || !dev_flag || (R > 0 && !idx)) return COMBO_ERR_INVALID_ARG;
+    DeviceInfo* dev = nullptr;
+    combo_status rc = device_info(&dev);
+    if (rc != COMBO_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(dev_flag, 0, sizeof(int32_t), st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    if (R == 0) return COMBO_OK;
+    const long long total = (long long)N * S * R;
+    long long blocks = (total + 255) / 256;
+    if (blocks > dev->sms * 8) blocks = dev->sms * 8;
+    combo::k_validate_idx<<<(int)blocks, 256, 0, st>>>(idx, N, S, R, dev_flag);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "validate_idx launch");
+    return COMBO_OK;
+}
+
+combo_status combo_round_host(const void* h_params_in, const void* h_grads, float lr, void* h_params_out,
+                              int elem_bytes, const float* h_weights, uint64_t seed, uint32_t round, int rounds,
+                              int N, int64_t P, int S, int R, void* d_in, void* d_grads, void* d_out,
+                              float* d_weights, int32_t* d_idx, int32_t* h_idx_out, void* stream) {
+    if (!h_params_in || !h_params_out || !d_in || !d_out) return COMBO_ERR_INVALID_ARG;
+    if ((h_grads != nullptr) != (d_grads != nullptr)) return COMBO_ERR_INVALID_ARG;
+    if (h_weights && !d_weights) return COMBO_ERR_INVALID_ARG;
+    if (elem_bytes != 4 && elem_bytes != 2) return COMBO_ERR_INVALID_ARG;
+    if (N < 1 || P < 1 || R < 0 || rounds < 1 || (R > 0 && !d_idx)) return COMBO_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bytes = (size_t)N * (size_t)P * (size_t)elem_bytes;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(d_in, h_params_in, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return cuda_fail(e, "copy params to device");
+    if (h_grads && (e = cudaMemcpyAsync(d_grads, h_grads, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return cuda_fail(e, "copy grads to device");
+    if (h_weights &&
+        (e = cudaMemcpyAsync(d_weights, h_weights, sizeof(float) * (size_t)N, cudaMemcpyHostToDevice, st)) !=
+            cudaSuccess)
+        return cuda_fail(e, "copy weights to device");
+    void* cur = d_in;
+    void* nxt = d_out;
+    for (int t = 0; t < rounds; ++t) {
+        combo_status rc = select_peers_impl(seed, round + (uint32_t)t, N, S, R, d_idx, st);
+        if (rc != COMBO_OK) return rc;
+        rc = aggregate_cols(cur, d_grads, lr, nxt, elem_bytes, h_weights ? d_weights : nullptr, d_idx, N, P, S, R,
+                            0, P, P, stream);
+        if (rc != COMBO_OK) return rc;
+        void* sw = cur; cur = nxt; nxt = sw;
+    }
+    if ((e = cudaMemcpyAsync(h_params_out, cur, bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return cuda_fail(e, "copy result to host");
+    if (h_idx_out && R > 0 &&
+        (e = cudaMemcpyAsync(h_idx_out, d_idx, sizeof(int32_t) * (size_t)N * S * R, cudaMemcpyDeviceToHost, st)) !=
+            cudaSuccess)
+        return cuda_fail(e, "copy idx to host");
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    return COMBO_OK;
+}
+
+combo_status combo_device_status(void) {
+    int v = 0;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+    if ((e = cudaMemcpyFromSymbol(&v, combo::g_dev_status, sizeof(int))) != cudaSuccess)
+        return cuda_fail(e, "cudaMemcpyFromSymbol");
+    if (v != 0) {
+        int zero = 0;
+        cudaMemcpyToSymbol(combo::g_dev_status, &zero, sizeof(int));
+        snprintf(t_cuda_err, sizeof(t_cuda_err), "bounded wait gave up at site %d", v);
+        return COMBO_ERR_DEVICE_TIMEOUT;
+    }
+    return COMBO_OK;
+}
+
+int combo_last_kernel_path(void) { return t_last_path; }
+
+void combo_set_kernel_path(int path) { t_force_path = (path == 1 || path == 2) ? path : 0; }
+
+void combo_set_tuning(int tile_elems, int stages) {
+    t_tile = tile_elems > 0 ? tile_elems : 0;
+    t_stages = stages > 0 ? stages : 0;
+}
+
+const char* combo_status_string(combo_status status) {
+    switch (status) {
+        case COMBO_OK: return "ok";
+        case COMBO_ERR_INVALID_ARG: return "invalid argument";
+        case COMBO_ERR_ALIAS: return "input and output overlap";
+        case COMBO_ERR_UNSUPPORTED: return "device is not compute capability 10.x";
+        case COMBO_ERR_CUDA: return "CUDA error";
+        case COMBO_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        default: return "unknown status";
+    }
+}
+
+const char* combo_last_cuda_error(void) { return t_cuda_err; }
+
+int combo_version(void) { return 100; }
+
+}  // extern "C"

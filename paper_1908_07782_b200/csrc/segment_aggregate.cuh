@@ -1,0 +1,517 @@
+// Segment-wise aggregation kernels (Eq. 3 and Eq. 4), all workers at once.
+//
+// Eq. 3 couples workers only at equal column p, and the peer table depends on
+// (worker, segment) alone.  The unit of work is therefore a column tile taken
+// through ALL N rows: the N x T block is brought from HBM into shared memory
+// once (one bulk async copy per row, completion counted on an mbarrier), every
+// worker's output for those columns is formed from it (R+1 shared-memory reads
+// per output element instead of R+1 HBM/L2 reads), and the N x T result goes
+// out with streaming 128-bit stores.  HBM traffic is then the compulsory one:
+// each worker-parameter read once and written once.
+//
+//   k_staged  persistent CTAs, 1 producer warp + 16 consumer warps, a ring of
+//             stages; warp-per-row accumulation in binary32
+//   k_direct  plain gather from global memory (any R, any N, tiny segments);
+//             also the "naive (R+1)-reads" contrast case for profiling
+//
+// Row alignment.  The ABI fixes dense [N][pitch] arrays, so a row starts at
+// byte (w*pitch*e) mod 16 =: phase.  Output vectors are aligned per OUTPUT row
+// (group g of row w covers columns [g*V - a_w, g*V - a_w + V), a_w = phase/e);
+// input rows are staged as the 16-byte aligned superset of the tile and read
+// back at the granule their phase difference allows (16, 4 or 2 bytes).  When
+// phases differ, a tile also loads V columns to the left of its nominal start
+// so that every group lies in exactly one tile.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace combo {
+
+// device status word: 0, or the code of the first bounded wait that gave up
+__device__ int g_dev_status;
+
+constexpr int kConsumerWarps = 16;
+constexpr int kConsumerThreads = 32 * kConsumerWarps;
+constexpr int kStagedThreads = 32 + kConsumerThreads;
+constexpr int kMaxStages = 8;
+constexpr int kStagedMaxR = 8;
+constexpr uint32_t kWaitCap = 1u << 24;   // polls before a wait is declared dead
+
+struct AggParams {
+    const unsigned char* in;
+    const unsigned char* grads;
+    unsigned char* out;
+    const float* weights;
+    const int32_t* idx;
+    long long pitch;     // elements between rows
+    long long p_begin;   // global column of local column 0
+    long long width;     // local columns
+    long long L;         // segment length of the whole vector
+    long long n_tiles;
+    long long arr_end_al;  // last valid byte of an input array, rounded down to 16
+    int N, S, R;
+    float lr;
+    int T;               // tile width in elements
+    int halo;            // extra columns loaded left of a tile (0 or V)
+    int stages;
+    int row_bytes;       // shared-memory bytes per staged row
+    unsigned tab_off;    // byte offset of the coefficient table in shared memory
+    unsigned stage_off;  // byte offset of stage 0
+    unsigned stage_bytes;
+};
+
+// ---------------------------------------------------------------- small helpers
+__device__ __forceinline__ float bf16_widen(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // round to nearest even
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int EB> struct ElemOps;
+template <> struct ElemOps<4> {
+    static constexpr int V = 4;
+    __device__ static __forceinline__ float load(const void* p) { return *reinterpret_cast<const float*>(p); }
+    __device__ static __forceinline__ void store(void* p, float v) { __stcs(reinterpret_cast<float*>(p), v); }
+    __device__ static __forceinline__ void store_vec(void* p, const float (&a)[4]) {
+        __stcs(reinterpret_cast<float4*>(p), make_float4(a[0], a[1], a[2], a[3]));
+    }
+};
+template <> struct ElemOps<2> {
+    static constexpr int V = 8;
+    __device__ static __forceinline__ float load(const void* p) {
+        return bf16_widen(*reinterpret_cast<const uint16_t*>(p));
+    }
+    __device__ static __forceinline__ void store(void* p, float v) {
+        __stcs(reinterpret_cast<unsigned short*>(p), (unsigned short)(pack_bf16x2_rn(v, 0.0f) & 0xffffu));
+    }
+    __device__ static __forceinline__ void store_vec(void* p, const float (&a)[8]) {
+        __stcs(reinterpret_cast<uint4*>(p),
+               make_uint4(pack_bf16x2_rn(a[0], a[1]), pack_bf16x2_rn(a[2], a[3]),
+                          pack_bf16x2_rn(a[4], a[5]), pack_bf16x2_rn(a[6], a[7])));
+    }
+};
+
+// Reads one output-aligned group (16 bytes of elements) at granule GB.
+template <int EB, int GB> struct GroupLoad;
+template <> struct GroupLoad<4, 16> {
+    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[4]) {
+        float4 v = *reinterpret_cast<const float4*>(p);
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    }
+};
+template <> struct GroupLoad<4, 4> {
+    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[4]) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) x[i] = reinterpret_cast<const float*>(p)[i];
+    }
+};
+template <> struct GroupLoad<2, 16> {
+    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8]) {
+        uint4 v = *reinterpret_cast<const uint4*>(p);
+        x[0] = bf16_widen(v.x & 0xffffu); x[1] = __uint_as_float(v.x & 0xffff0000u);
+        x[2] = bf16_widen(v.y & 0xffffu); x[3] = __uint_as_float(v.y & 0xffff0000u);
+        x[4] = bf16_widen(v.z & 0xffffu); x[5] = __uint_as_float(v.z & 0xffff0000u);
+        x[6] = bf16_widen(v.w & 0xffffu); x[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+};
+template <> struct GroupLoad<2, 4> {
+    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8]) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t v = reinterpret_cast<const uint32_t*>(p)[i];
+            x[2 * i] = bf16_widen(v & 0xffffu);
+            x[2 * i + 1] = __uint_as_float(v & 0xffff0000u);
+        }
+    }
+};
+template <> struct GroupLoad<2, 2> {
+    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8]) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = bf16_widen(reinterpret_cast<const uint16_t*>(p)[i]);
+    }
+};
+
+// Coefficients of Eq. 3 for one (worker, segment): c_j = |D_j| / sum over P_l,
+// provider order self, then peers ascending.  cf[0..R], binary32.
+__device__ __forceinline__ void eq3_coefficients(const float* __restrict__ weights,
+                                                 const int32_t* __restrict__ peers, int w, int R,
+                                                 float* cf) {
+    const float dw = weights ? weights[w] : 1.0f;
+    float den = dw;
+    for (int r = 0; r < R; ++r) den = __fadd_rn(den, weights ? weights[peers[r]] : 1.0f);
+    cf[0] = __fdiv_rn(dw, den);
+    for (int r = 0; r < R; ++r) cf[r + 1] = __fdiv_rn(weights ? weights[peers[r]] : 1.0f, den);
+}
+
+// ---------------------------------------------------------------- direct gather
+template <int EB, bool SGD>
+__device__ __forceinline__ float direct_x(const AggParams& p, int k, long long c) {
+    const size_t off = ((size_t)k * (size_t)p.pitch + (size_t)c) * EB;
+    float x = ElemOps<EB>::load(p.in + off);
+    if (SGD) x = fmaf(-p.lr, ElemOps<EB>::load(p.grads + off), x);
+    return x;
+}
+
+template <int EB, bool SGD>
+__global__ void __launch_bounds__(256) k_direct(const AggParams p) {
+    constexpr int V = ElemOps<EB>::V;
+    const long long G = (p.width + V - 1) / V + 1;      // groups per row, phase spill included
+    const long long items = G * (long long)p.N;
+    const bool rows_aligned = (p.pitch % V) == 0;
+    for (long long it = blockIdx.x * 256LL + threadIdx.x; it < items; it += (long long)gridDim.x * 256LL) {
+        const int w = (int)(it / G);
+        const long long g = it - (long long)w * G;
+        const int a_w = (int)(((long long)w * p.pitch) & (V - 1));
+        const long long c0 = g * V - a_w;
+        const long long lo = c0 < 0 ? 0 : c0;
+        const long long hi = (c0 + V > p.width) ? p.width : c0 + V;
+        if (lo >= hi) continue;
+        const long long l_lo = (p.p_begin + lo) / p.L, l_hi = (p.p_begin + hi - 1) / p.L;
+        if (hi - lo == V && l_lo == l_hi && rows_aligned) {
+            const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l_lo) * (size_t)p.R;
+            const float dw = p.weights ? p.weights[w] : 1.0f;
+            float den = dw;
+            for (int r = 0; r < p.R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+            float acc[V], x[V];
+            {
+                const size_t off = ((size_t)w * (size_t)p.pitch + (size_t)c0) * EB;
+                GroupLoad<EB, 16>::run(p.in + off, x);
+                if (SGD) {
+                    float gx[V];
+                    GroupLoad<EB, 16>::run(p.grads + off, gx);
+#pragma unroll
+                    for (int i = 0; i < V; ++i) x[i] = fmaf(-p.lr, gx[i], x[i]);
+                }
+                const float c = __fdiv_rn(dw, den);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(c, x[i]);
+            }
+            for (int r = 0; r < p.R; ++r) {
+                const int k = peers[r];
+                const size_t off = ((size_t)k * (size_t)p.pitch + (size_t)c0) * EB;
+                GroupLoad<EB, 16>::run(p.in + off, x);
+                if (SGD) {
+                    float gx[V];
+                    GroupLoad<EB, 16>::run(p.grads + off, gx);
+#pragma unroll
+                    for (int i = 0; i < V; ++i) x[i] = fmaf(-p.lr, gx[i], x[i]);
+                }
+                const float c = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] = fmaf(c, x[i], acc[i]);
+            }
+            ElemOps<EB>::store_vec(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c0) * EB, acc);
+        } else {
+            for (long long c = lo; c < hi; ++c) {
+                const long long l = (p.p_begin + c) / p.L;
+                const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)p.R;
+                const float dw = p.weights ? p.weights[w] : 1.0f;
+                float den = dw;
+                for (int r = 0; r < p.R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+                float acc = __fmul_rn(__fdiv_rn(dw, den), direct_x<EB, SGD>(p, w, c));
+                for (int r = 0; r < p.R; ++r) {
+                    const int k = peers[r];
+                    acc = fmaf(__fdiv_rn(p.weights ? p.weights[k] : 1.0f, den), direct_x<EB, SGD>(p, k, c), acc);
+                }
+                ElemOps<EB>::store(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c) * EB, acc);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- mbarrier / bulk copy (PTX)
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar),
+                 "r"(bytes)
+                 : "memory");
+}
+// Bounded wait: false when the phase did not complete within kWaitCap polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kWaitCap; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (it > 4096) __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
+struct TileMeta {
+    long long cs;    // first local column held in the stage
+    long long ce;    // one past the last
+    long long bnd;   // local column where segment l0+1 starts
+    int l0;          // segment of column cs
+    int pad;
+};
+
+// shared-memory header: barriers and per-stage metadata
+struct StagedHeader {
+    unsigned long long full[kMaxStages];
+    unsigned long long empty[kMaxStages];
+    unsigned long long csync;            // consumer-wide barrier (16 arrivals)
+    unsigned long long pad;
+    TileMeta meta[kMaxStages];
+};
+
+__device__ __forceinline__ void staged_fail(int code) { atomicCAS(&g_dev_status, 0, code); }
+
+// Consumer-wide barrier with a bounded wait (all 16 consumer warps).
+__device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t& phase, int lane) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+    bool ok = mbar_wait(bar, phase & 1u);
+    phase ^= 1u;
+    return ok;
+}
+
+template <int EB, int GB, bool SGD, int RT>
+__global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p) {
+    constexpr int V = ElemOps<EB>::V;
+    constexpr int RMAX = (RT >= 0) ? RT : kStagedMaxR;
+    extern __shared__ __align__(128) unsigned char smem[];
+    StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int N = p.N, R = (RT >= 0) ? RT : p.R;
+    const int stages = p.stages;
+    const int narr = SGD ? 2 : 1;
+
+    int32_t* tab_peer = reinterpret_cast<int32_t*>(smem + p.tab_off);           // [2][N][R]
+    float* tab_coef = reinterpret_cast<float*>(tab_peer + 2 * N * (R > 0 ? R : 1));  // [2][N][R+1]
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(smem_u32(&hdr->full[s]), 1);
+            mbar_init(smem_u32(&hdr->empty[s]), kConsumerWarps);
+        }
+        mbar_init(smem_u32(&hdr->csync), kConsumerWarps);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        long long n = 0;
+        bool alive = true;
+        for (long long tile = blockIdx.x; tile < p.n_tiles && alive; tile += gridDim.x, ++n) {
+            const int s = (int)(n % stages);
+            const uint32_t ph = (uint32_t)((n / stages) & 1);
+            if (!mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); alive = false; break; }
+            long long cs = tile * p.T - p.halo; if (cs < 0) cs = 0;
+            long long ce = (tile + 1) * p.T; if (ce > p.width) ce = p.width;
+            unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
+            uint32_t my_bytes = 0;
+            for (int k = lane; k < N; k += 32) {
+                const long long b0 = ((long long)k * p.pitch + cs) * EB;
+                const long long b1 = ((long long)k * p.pitch + ce) * EB;
+                const long long A = b0 & ~15LL;
+                long long E = (b1 + 15) & ~15LL;
+                if (E > p.arr_end_al) E = p.arr_end_al;
+                if (E < A) E = A;
+                my_bytes += (uint32_t)(E - A) * narr;
+                if (E < b1) {
+                    // the array ends inside this 16-byte granule: fetch the last elements by hand
+                    for (int a = 0; a < narr; ++a) {
+                        const unsigned char* src = (a == 0 ? p.in : p.grads);
+                        unsigned char* dst = stage + ((size_t)a * N + k) * p.row_bytes;
+                        for (long long b = (E > b0 ? E : b0); b < b1; b += EB) {
+                            if (EB == 4) *reinterpret_cast<uint32_t*>(dst + (b - A)) = *reinterpret_cast<const uint32_t*>(src + b);
+                            else *reinterpret_cast<uint16_t*>(dst + (b - A)) = *reinterpret_cast<const uint16_t*>(src + b);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) my_bytes += __shfl_xor_sync(0xffffffffu, my_bytes, o);
+            if (lane == 0) {
+                TileMeta& m = hdr->meta[s];
+                const int l0 = (int)((p.p_begin + cs) / p.L);
+                m.cs = cs; m.ce = ce; m.l0 = l0;
+                m.bnd = (long long)(l0 + 1) * p.L - p.p_begin;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_expect_tx(smem_u32(&hdr->full[s]), my_bytes);
+            __syncwarp();
+            const uint32_t bar = smem_u32(&hdr->full[s]);
+            for (int k = lane; k < N; k += 32) {
+                const long long b0 = ((long long)k * p.pitch + cs) * EB;
+                const long long b1 = ((long long)k * p.pitch + ce) * EB;
+                const long long A = b0 & ~15LL;
+                long long E = (b1 + 15) & ~15LL;
+                if (E > p.arr_end_al) E = p.arr_end_al;
+                if (E > A) {
+                    bulk_g2s(smem_u32(stage + (size_t)k * p.row_bytes), p.in + A, (uint32_t)(E - A), bar);
+                    if (SGD)
+                        bulk_g2s(smem_u32(stage + ((size_t)N + k) * p.row_bytes), p.grads + A, (uint32_t)(E - A), bar);
+                }
+            }
+        }
+        // Leave last: every stage this warp armed must have landed before the CTA's
+        // shared memory can be released, even if the consumers gave up.
+        if (lane == 0) {
+            const long long first = n > stages ? n - stages : 0;
+            for (long long q = first; q < n; ++q) {
+                const int s = (int)(q % stages);
+                if (!mbar_wait(smem_u32(&hdr->full[s]), (uint32_t)((q / stages) & 1))) staged_fail(2);
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- consumers
+    const int cw = warp - 1;
+    const int ctid = tid - 32;
+    uint32_t csync_phase = 0;
+    int cached_l0 = -1;
+    const int GT = p.T / V;          // groups per tile
+    const int CH = GT / 32;          // 32-group chunks per row per tile
+    const int n_items = N * CH;
+    const int ipw = (n_items + kConsumerWarps - 1) / kConsumerWarps;
+    const uint32_t csync = smem_u32(&hdr->csync);
+
+    long long n = 0;
+    for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
+        const int s = (int)(n % stages);
+        const uint32_t ph = (uint32_t)((n / stages) & 1);
+        if (!mbar_wait(smem_u32(&hdr->full[s]), ph)) { staged_fail(3); return; }
+        const TileMeta m = hdr->meta[s];
+        unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
+
+        if (m.l0 != cached_l0) {
+            // coefficient / peer table for segments l0 and l0+1 (rebuilt at most S times per CTA)
+            if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(4); return; }
+            for (int q = ctid; q < 2 * N; q += kConsumerThreads) {
+                const int slot = q / N, w = q - slot * N;
+                const int l = m.l0 + slot;
+                if (l < p.S) {
+                    const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
+                    float cf[RMAX + 1];
+                    const float dw = p.weights ? p.weights[w] : 1.0f;
+                    float den = dw;
+#pragma unroll
+                    for (int r = 0; r < RMAX; ++r)
+                        if (r < R) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+                    cf[0] = __fdiv_rn(dw, den);
+#pragma unroll
+                    for (int r = 0; r < RMAX; ++r)
+                        if (r < R) cf[r + 1] = __fdiv_rn(p.weights ? p.weights[peers[r]] : 1.0f, den);
+                    float* tc = tab_coef + ((size_t)slot * N + w) * (R + 1);
+                    int32_t* tp = tab_peer + ((size_t)slot * N + w) * (R > 0 ? R : 1);
+                    tc[0] = cf[0];
+#pragma unroll
+                    for (int r = 0; r < RMAX; ++r)
+                        if (r < R) { tc[r + 1] = cf[r + 1]; tp[r] = peers[r]; }
+                }
+            }
+            if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
+            cached_l0 = m.l0;
+        }
+
+        if (SGD) {
+            // local step on the staged tile, in place: x <- fma(-lr, g, x), every row
+            const int nvec = N * p.row_bytes / 16;
+            float4* xs = reinterpret_cast<float4*>(stage);
+            const float4* gs = reinterpret_cast<const float4*>(stage + (size_t)N * p.row_bytes);
+            const float nlr = -p.lr;
+            for (int v = ctid; v < nvec; v += kConsumerThreads) {
+                float4 x = xs[v];
+                const float4 g = gs[v];
+                x.x = fmaf(nlr, g.x, x.x); x.y = fmaf(nlr, g.y, x.y);
+                x.z = fmaf(nlr, g.z, x.z); x.w = fmaf(nlr, g.w, x.w);
+                xs[v] = x;
+            }
+            if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(6); return; }
+        }
+
+        const bool has_bnd = m.bnd < m.ce;     // a segment boundary lies inside the staged columns
+        const long long g_tile0 = tile * (long long)GT;
+
+        int cur_row = -1;
+        int a_w = 0;
+        float cf[RMAX + 1];
+        int poff[RMAX + 1];
+        const int it_end = (cw + 1) * ipw < n_items ? (cw + 1) * ipw : n_items;
+        int row = (cw * ipw) / CH;
+        int chunk = (cw * ipw) - row * CH;
+        for (int item = cw * ipw; item < it_end; ++item) {
+            if (row != cur_row) {
+                cur_row = row;
+                a_w = (int)(((long long)row * p.pitch) & (V - 1));
+                if (!has_bnd) {
+                    const float* tc = tab_coef + (size_t)row * (R + 1);
+                    const int32_t* tp = tab_peer + (size_t)row * (R > 0 ? R : 1);
+                    cf[0] = tc[0];
+                    poff[0] = row * p.row_bytes;
+#pragma unroll
+                    for (int r = 0; r < RMAX; ++r)
+                        if (r < R) {
+                            const int k = tp[r];
+                            const int a_k = (int)(((long long)k * p.pitch) & (V - 1));
+                            cf[r + 1] = tc[r + 1];
+                            poff[r + 1] = k * p.row_bytes + (a_k - a_w) * EB;
+                        }
+                }
+            }
+            const long long g = g_tile0 + chunk * 32 + lane;
+            const long long c0 = g * V - a_w;
+            const bool full = (c0 >= 0) && (c0 + V <= p.width);
+            if (full && !has_bnd) {
+                const int goff = (int)(g * V - m.cs) * EB;
+                float acc[V], x[V];
+                GroupLoad<EB, GB>::run(stage + poff[0] + goff, x);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(cf[0], x[i]);
+#pragma unroll
+                for (int r = 0; r < RMAX; ++r)
+                    if (r < R) {
+                        GroupLoad<EB, GB>::run(stage + poff[r + 1] + goff, x);
+#pragma unroll
+                        for (int i = 0; i < V; ++i) acc[i] = fmaf(cf[r + 1], x[i], acc[i]);
+                    }
+                ElemOps<EB>::store_vec(p.out + ((size_t)row * (size_t)p.pitch + (size_t)c0) * EB, acc);
+            } else {
+                // edge of the row or a tile that holds a segment boundary: element by element
+                const long long lo = c0 < 0 ? 0 : c0;
+                const long long hi = (c0 + V > p.width) ? p.width : c0 + V;
+                for (long long c = lo; c < hi; ++c) {
+                    const int slot = (c >= m.bnd) ? 1 : 0;
+                    const float* tc = tab_coef + ((size_t)slot * N + row) * (R + 1);
+                    const int32_t* tp = tab_peer + ((size_t)slot * N + row) * (R > 0 ? R : 1);
+                    const int eoff = (int)(c - m.cs) * EB;
+                    float acc = __fmul_rn(tc[0], ElemOps<EB>::load(stage + row * p.row_bytes + a_w * EB + eoff));
+                    for (int r = 0; r < R; ++r) {
+                        const int k = tp[r];
+                        const int a_k = (int)(((long long)k * p.pitch) & (V - 1));
+                        acc = fmaf(tc[r + 1], ElemOps<EB>::load(stage + k * p.row_bytes + a_k * EB + eoff), acc);
+                    }
+                    ElemOps<EB>::store(p.out + ((size_t)row * (size_t)p.pitch + (size_t)c) * EB, acc);
+                }
+            }
+            if (++chunk == CH) { chunk = 0; ++row; }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
+    }
+}
+
+}  // namespace combo

@@ -1,0 +1,118 @@
+// Peer selection kernel (Section 4.1 step 2, "Segments Pulling").
+//
+// One CTA per worker.  The random draw positions of a shuffle are a pure
+// function of (seed, round, worker, epoch, position), so all threads compute
+// them in parallel; the swaps themselves are inherently sequential and are
+// applied by one lane.  The peers of the segment being filled are kept as a
+// byte map over worker ids, which serves both the "skip what this segment
+// already holds" rule after a refill and the ascending output order.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace combo {
+
+// splitmix64 output function (Steele, Lea, Flood 2014) and its increment.
+__device__ __forceinline__ uint64_t splitmix_out(uint64_t z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+__device__ __forceinline__ uint64_t splitmix_step(uint64_t state) {
+    return splitmix_out(state + 0x9E3779B97F4A7C15ull);
+}
+
+constexpr int kSelectThreads = 128;
+
+__host__ __device__ inline size_t select_peers_smem_bytes(int N) {
+    // perm[N-1] + aux[N-1] as int32, mark[N] as bytes, rounded up
+    return (size_t)(N > 1 ? N - 1 : 1) * 8 + (size_t)N + 16;
+}
+
+__global__ void __launch_bounds__(kSelectThreads)
+k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __restrict__ idx) {
+    extern __shared__ __align__(16) unsigned char sp_smem[];
+    const int w = blockIdx.x;
+    const int M = N - 1;
+    int32_t* perm = reinterpret_cast<int32_t*>(sp_smem);
+    int32_t* aux = perm + M;
+    uint8_t* mark = reinterpret_cast<uint8_t*>(aux + M);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    for (int v = tid; v < N; v += kSelectThreads) mark[v] = 0;
+
+    // chain: seed -> (round | worker) -> (epoch | position)
+    uint64_t hw = splitmix_step(seed);
+    hw = splitmix_step(hw ^ (((uint64_t)round << 32) | (uint64_t)(uint32_t)w));
+
+    const long long total = (long long)S * (long long)R;
+    const uint32_t epochs = (uint32_t)((total + M - 1) / M);
+    long long done = 0, row = 0;   // warp-0 uniform
+    int nc = 0;                    // peers the current segment holds so far
+
+    for (uint32_t e = 0; e < epochs; ++e) {
+        for (int t = 1 + tid; t < M; t += kSelectThreads) {
+            uint64_t h = splitmix_step(hw ^ (((uint64_t)e << 32) | (uint64_t)(uint32_t)t));
+            aux[t] = (int32_t)(((h >> 32) * (uint64_t)(t + 1)) >> 32);   // in [0, t]
+        }
+        for (int i = tid; i < M; i += kSelectThreads) perm[i] = i + (i >= w ? 1 : 0);
+        __syncthreads();
+        if (warp == 0) {
+            if (lane == 0) {
+                for (int t = M - 1; t >= 1; --t) {          // Fisher-Yates
+                    int j = aux[t];
+                    int32_t a = perm[t]; perm[t] = perm[j]; perm[j] = a;
+                }
+                if (nc > 0) {                                // held peers go last, order kept
+                    int a = 0;
+                    for (int i = 0; i < M; ++i) if (!mark[perm[i]]) aux[a++] = perm[i];
+                    for (int i = 0; i < M; ++i) if (mark[perm[i]]) aux[a++] = perm[i];
+                    for (int i = 0; i < M; ++i) perm[i] = aux[i];
+                }
+            }
+            __syncwarp();
+            int pos = 0;
+            while (pos < M && done < total) {
+                int take = R - nc;
+                if (take > M - pos) take = M - pos;
+                for (int i = lane; i < take; i += 32) mark[perm[pos + i]] = 1;
+                pos += take; nc += take; done += take;
+                __syncwarp();
+                if (nc == R) {                               // emit the row ascending
+                    int32_t* out = idx + (size_t)((long long)w * S + row) * (size_t)R;
+                    int k = 0;
+                    for (int v0 = 0; v0 < N; v0 += 32) {
+                        int v = v0 + lane;
+                        bool bit = (v < N) && mark[v];
+                        unsigned b = __ballot_sync(0xffffffffu, bit);
+                        if (bit) {
+                            out[k + __popc(b & ((1u << lane) - 1u))] = v;
+                            mark[v] = 0;
+                        }
+                        k += __popc(b);
+                    }
+                    __syncwarp();
+                    nc = 0;
+                    ++row;
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// Checks an idx table: range, never self, strictly ascending rows.
+__global__ void k_validate_idx(const int32_t* __restrict__ idx, int N, int S, int R,
+                               int32_t* __restrict__ flag) {
+    long long total = (long long)N * S * R;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        int r = (int)(i % R);
+        int w = (int)(i / ((long long)S * R));
+        int v = idx[i];
+        bool bad = v < 0 || v >= N || v == w || (r > 0 && idx[i - 1] >= v);
+        if (bad) atomicCAS(flag, 0, (int32_t)(i < 0x7ffffffeLL ? i + 1 : 0x7fffffff));
+    }
+}
+
+}  // namespace combo

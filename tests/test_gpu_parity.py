@@ -1,0 +1,247 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1908_07782_b200 as combo
+from paper_1908_07782_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import DEV, check_against_oracle, gpu_aggregate, gpu_select, to_bits  # noqa: E402
+
+
+# ------------------------------------------------------------------ peer sampler
+SAMPLER_CASES = [
+    (8, 4, 2), (32, 8, 3), (64, 10, 4), (128, 16, 4), (16, 32, 4),      # the five workloads
+    (2, 1, 1), (2, 5, 1), (3, 7, 2), (4, 2, 2), (5, 4, 1), (5, 9, 4), (9, 3, 8), (33, 2, 32),
+    (130, 3, 1), (300, 5, 7), (257, 2, 256), (1000, 2, 999), (4097, 3, 5), (1, 4, 0), (6, 3, 0),
+]
+
+
+@pytest.mark.parametrize("N,S,R", SAMPLER_CASES)
+def test_select_peers_bit_exact(N, S, R):
+    for seed, rnd in ((1, 0), (1, 7), (0xDEADBEEFCAFEF00D, 4_000_000_000)):
+        got = gpu_select(seed, rnd, N, S, R).cpu().numpy()
+        want = oracle.select_peers(seed, rnd, N, S, R)
+        assert got.shape == want.shape
+        assert (got == want).all()
+
+
+def test_select_peers_default_stream_entry():
+    idx = torch.zeros((8, 4, 2), dtype=torch.int32, device=DEV)
+    combo.combo_select_peers_default_stream(1, 0, 8, 4, 2, idx)
+    torch.cuda.synchronize()
+    assert (idx.cpu().numpy() == oracle.select_peers(1, 0, 8, 4, 2)).all()
+
+
+def test_select_peers_rounds_of_every_workload():
+    for name, wl in synth.WORKLOADS.items():
+        for rnd in range(wl.rounds):
+            got = gpu_select(wl.sampler_seed, rnd, wl.N, wl.S, wl.R).cpu().numpy()
+            assert (got == oracle.select_peers(wl.sampler_seed, rnd, wl.N, wl.S, wl.R)).all(), name
+
+
+def test_validate_idx():
+    N, S, R = 16, 4, 3
+    idx = gpu_select(1, 0, N, S, R)
+    flag = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+    combo.combo_validate_idx(idx, N, S, R, flag)
+    assert int(flag.item()) == 0
+    for pos, val in ((5, 0), (7, N), (9, -1)):
+        bad = idx.clone().view(-1)
+        if pos == 5:
+            bad[pos] = pos // (S * R)          # the worker itself
+        else:
+            bad[pos] = val
+        combo.combo_validate_idx(bad, N, S, R, flag)
+        assert int(flag.item()) != 0
+    bad = idx.clone()
+    bad[3, 2, 1] = bad[3, 2, 0]                # repeated peer
+    combo.combo_validate_idx(bad, N, S, R, flag)
+    assert int(flag.item()) != 0
+
+
+# ------------------------------------------------------------------ aggregation, small sweep
+def _inputs(N, P, dtype, seed, sigma=0.05):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    x = (torch.randn(N, P, generator=g) * sigma).to(dtype).to(DEV)
+    grads = (torch.randn(N, P, generator=g) * 1e-3).to(DEV)
+    counts = torch.randint(500, 1501, (N,), generator=g).float().to(DEV)
+    return x, grads, counts
+
+
+SMALL = [(N, P, S, R) for N in (1, 2, 3, 5, 8) for P in (1, 2, 3, 7, 8, 9, 31, 64, 70, 257)
+         for S in (1, 2, 3, 9) for R in (0, 1, 2, 4, 7) if R <= N - 1]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_aggregate_tiny_shapes_exhaustive(dtype):
+    # every small P (odd alignments, P < S with empty segments), both kernels where they apply
+    for (N, P, S, R) in SMALL:
+        x, grads, counts = _inputs(N, P, dtype, N * 131 + P)
+        idx_np = oracle.select_peers(3, 1, N, S, R)
+        idx = torch.from_numpy(idx_np).to(DEV)
+        for weights in (None, counts):
+            out, used = gpu_aggregate(x, idx, S, R, weights=weights)
+            assert used == combo.PATH_DIRECT
+            check_against_oracle(x, out, idx_np, S, R, weights=weights)
+        if dtype == torch.float32:
+            out, _ = gpu_aggregate(x, idx, S, R, grads=grads, lr=0.01)
+            check_against_oracle(x, out, idx_np, S, R, grads=grads, lr=0.01)
+
+
+MEDIUM = [
+    # N, P, S, R, dtype, weighted
+    (8, 40_000, 4, 2, torch.float32, False),
+    (8, 40_001, 4, 2, torch.float32, True),       # rows not 16-byte aligned (fp32, granule 4)
+    (32, 20_003, 8, 3, torch.float32, True),
+    (32, 20_004, 8, 3, torch.float32, True),      # odd segment length, aligned rows
+    (64, 9_992, 10, 4, torch.float32, False),     # last segment shorter
+    (16, 33_000, 32, 4, torch.float32, False),
+    (5, 50_000, 3, 4, torch.float32, True),       # R = N-1
+    (12, 30_000, 5, 8, torch.float32, True),      # largest R the staged kernel takes
+    (12, 30_000, 5, 9, torch.float32, True),      # beyond it: direct kernel
+    (7, 30_000, 3, 0, torch.float32, False),      # R = 0
+    (1, 30_000, 3, 0, torch.float32, False),      # a single worker
+    (128, 5_002, 16, 4, torch.bfloat16, False),   # row pitch = 4 mod 16 bytes (granule 4)
+    (128, 5_003, 16, 4, torch.bfloat16, True),    # odd pitch (granule 2)
+    (128, 5_120, 16, 4, torch.bfloat16, False),   # aligned rows
+    (20, 20_000, 7, 3, torch.bfloat16, True),
+    (9, 70_001, 2, 2, torch.bfloat16, False),
+]
+
+
+@pytest.mark.parametrize("N,P,S,R,dtype,weighted", MEDIUM)
+@pytest.mark.parametrize("path", [combo.PATH_DIRECT, combo.PATH_STAGED])
+def test_aggregate_medium_both_kernels(N, P, S, R, dtype, weighted, path):
+    x, grads, counts = _inputs(N, P, dtype, 17 * N + P % 1000)
+    weights = counts if weighted else None
+    idx_np = oracle.select_peers(1, 2, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV) if R > 0 else None
+    out, used = gpu_aggregate(x, idx, S, R, weights=weights, path=path)
+    if path == combo.PATH_STAGED and R <= 8:
+        assert used == combo.PATH_STAGED
+    check_against_oracle(x, out, idx_np, S, R, weights=weights)
+    if R == 0:
+        assert torch.equal(out, x)                                   # identity, bit for bit
+    if dtype == torch.float32:
+        out, _ = gpu_aggregate(x, idx, S, R, weights=weights, grads=grads, lr=0.01, path=path)
+        check_against_oracle(x, out, idx_np, S, R, weights=weights, grads=grads, lr=0.01)
+
+
+@pytest.mark.parametrize("tile,stages", [(128, 2), (128, 8), (256, 3), (1024, 2), (0, 0)])
+def test_staged_tile_shapes(tile, stages):
+    # many tiles per CTA, ragged last tile, segment boundaries inside tiles
+    N, P, S, R = 16, 1_000_003, 6, 3
+    x, grads, counts = _inputs(N, P, torch.float32, 5)
+    idx_np = oracle.select_peers(9, 0, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    combo.combo_set_tuning(tile, stages)
+    try:
+        out, used = gpu_aggregate(x, idx, S, R, weights=counts, path=combo.PATH_STAGED)
+        assert used == combo.PATH_STAGED
+        check_against_oracle(x, out, idx_np, S, R, weights=counts)
+        xb = x[:, :600_010].contiguous().to(torch.bfloat16)
+        t16 = tile if tile % 256 == 0 else 0
+        combo.combo_set_tuning(t16, stages)
+        outb, used = gpu_aggregate(xb, idx, S, R, path=combo.PATH_STAGED)
+        assert used == combo.PATH_STAGED
+        check_against_oracle(xb, outb, idx_np, S, R)
+    finally:
+        combo.combo_set_tuning(0, 0)
+
+
+def test_special_cases_on_device():
+    N, P, S = 6, 100_000, 4
+    x, _, counts = _inputs(N, P, torch.float32, 3)
+    # R = n-1: every worker gets the global weighted mean (the all-reduce result)
+    idx_np = oracle.select_peers(1, 0, N, S, N - 1)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    for path in (combo.PATH_DIRECT, combo.PATH_STAGED):
+        out, _ = gpu_aggregate(x, idx, S, N - 1, weights=counts, path=path)
+        mean = np.average(x.cpu().numpy().astype(np.float64), axis=0, weights=counts.cpu().numpy())
+        assert np.abs(out.cpu().numpy() - mean).max() <= 1e-6 * float(x.abs().max())
+        # identical inputs stay identical
+        same = x[:1].repeat(N, 1).contiguous()
+        out, _ = gpu_aggregate(same, idx, S, N - 1, weights=counts, path=path)
+        assert (out - same).abs().max().item() <= 1e-6 * float(x.abs().max())
+        # convexity
+        i2 = torch.from_numpy(oracle.select_peers(1, 0, N, S, 2)).to(DEV)
+        out, _ = gpu_aggregate(x, i2, S, 2, weights=counts, path=path)
+        assert (out <= x.max(dim=0).values + 1e-9).all() and (out >= x.min(dim=0).values - 1e-9).all()
+
+
+def test_argument_errors():
+    N, P, S, R = 4, 1000, 2, 1
+    x = torch.zeros(N, P, device=DEV)
+    out = torch.zeros(N, P, device=DEV)
+    idx = gpu_select(1, 0, N, S, R)
+    E = combo.ComboError
+    with pytest.raises(E) as e:
+        combo.combo_segment_aggregate(x, x, None, idx, N, P, S, R)
+    assert e.value.status == 2                                        # alias
+    both = torch.zeros(2 * N * P, device=DEV)
+    with pytest.raises(E) as e:
+        combo.combo_segment_aggregate(both[:N * P], both[N * P - 4:2 * N * P - 4], None, idx, N, P, S, R)
+    assert e.value.status == 2                                        # partial overlap
+    with pytest.raises(E) as e:
+        combo.combo_segment_aggregate(both[1:N * P + 1], out, None, idx, N, P, S, R)
+    assert e.value.status == 1                                        # misaligned base
+    for bad in ((0, P, S, R), (N, 0, S, R), (N, P, 0, R), (N, P, S, -1), (N, P, S, N)):
+        with pytest.raises(E) as e:
+            combo.combo_segment_aggregate(x, out, None, idx, *bad)
+        assert e.value.status == 1
+    with pytest.raises(E) as e:
+        combo.combo_segment_aggregate(x, out, None, None, N, P, S, R)
+    assert e.value.status == 1                                        # idx required when R > 0
+    with pytest.raises(E) as e:
+        combo.combo_select_peers(1, 0, 4, 2, 4, idx)
+    assert e.value.status == 1
+    combo.combo_device_status()
+
+
+def test_column_shards_need_no_exchange():
+    # two shards of the columns, each aggregated on its own, give the full result
+    N, P, S, R = 8, 120_000, 5, 2
+    x, grads, counts = _inputs(N, P, torch.float32, 11)
+    idx_np = oracle.select_peers(1, 0, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    full, _ = gpu_aggregate(x, idx, S, R, weights=counts)
+    cut = 50_004
+    for (a, b) in ((0, cut), (cut, P)):
+        shard = x[:, a:b].contiguous()
+        out = torch.empty_like(shard)
+        combo.combo_segment_aggregate_cols(shard, None, 0.0, out, 4, counts, idx, N, P, S, R, a, b - a,
+                                           b - a)
+        torch.cuda.synchronize()
+        assert torch.equal(out, full[:, a:b])
+        check_against_oracle(shard, out, idx_np, S, R, weights=counts, P=P, p_begin=a)
+
+
+def test_round_from_host_memory():
+    N, P, S, R = 8, 50_000, 4, 2
+    g = torch.Generator().manual_seed(1)
+    hx = (torch.randn(N, P, generator=g) * 0.05).pin_memory()
+    hw = torch.randint(500, 1501, (N,), generator=g).float()
+    hout = torch.empty_like(hx).pin_memory()
+    hidx = torch.empty((N, S, R), dtype=torch.int32).pin_memory()
+    d_in = torch.empty(N, P, device=DEV)
+    d_out = torch.empty(N, P, device=DEV)
+    d_w = torch.empty(N, device=DEV)
+    d_idx = torch.empty((N, S, R), dtype=torch.int32, device=DEV)
+    combo.combo_round_host(hx, None, 0.0, hout, 4, hw, 1, 3, 1, N, P, S, R, d_in, None, d_out, d_w, d_idx,
+                           hidx)
+    idx_np = oracle.select_peers(1, 3, N, S, R)
+    assert (hidx.numpy() == idx_np).all()
+    check_against_oracle(hx, hout, idx_np, S, R, weights=hw)
+    # three chained rounds: each round's input is the previous round's output
+    combo.combo_round_host(hx, None, 0.0, hout, 4, hw, 1, 3, 3, N, P, S, R, d_in, None, d_out, d_w, d_idx,
+                           hidx)
+    cur = hx.numpy()
+    for t in range(3):
+        idx_t = oracle.select_peers(1, 3 + t, N, S, R)
+        cur = oracle.segment_aggregate_ordered_f32(cur, idx_t, S, R, weights=hw.numpy())
+    assert (hidx.numpy() == idx_t).all()
+    assert (hout.numpy().view(np.uint32) == cur.view(np.uint32)).all()
