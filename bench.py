@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the segmented-gossip synchronization round on B200.
+
+One STEP = the workload's whole round sequence (peer selection + segment-wise
+aggregation, `rounds` times, ping-pong buffers) over one batch of synthetic
+parameters.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2] [--impl reference]
+
+N > 1 (launched with torch.distributed.run): every rank runs an independent
+federation replica on its own GPU (Eq. 3 needs no exchange between column
+shards or replicas), times are the max over ranks, the value is the sum of all
+ranks' worker-parameters over that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "worker_params_aggregated_per_s"
+UNIT = "worker-params/s"
+FALLBACK_HBM_GBS = 6650.0
+NCU_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic.json")
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="2", help="1..5 or a workload name (default: 2)")
+    ap.add_argument("--impl", default="combo", choices=["combo", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 direct gather, 2 staged")
+    ap.add_argument("--tile", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    return ap.parse_args()
+
+
+def elem_bytes(wl):
+    return 4 if wl.dtype == "f32" else 2
+
+
+def algorithmic_bytes_per_launch(wl):
+    """Compulsory HBM traffic of one aggregation launch: every worker-parameter
+    read once and written once (and its gradient read once when the local step
+    is fused)."""
+    e = elem_bytes(wl)
+    return wl.N * wl.P * e * 2 + (wl.N * wl.P * 4 if wl.fused_sgd else 0)
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            # samples under load: the upper half of the observed clocks
+            out["sm_mhz"] = statistics.median(sm)
+            out["sm_max_mhz"] = max(mx)
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------ reference arm (CPU oracle)
+def oracle_sample(wl, target_wp, rounds_hint=1):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload:
+    all N rows of a column slab.  Returns (worker-params/s, description, wp)."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_1908_07782_b200 import synth
+
+    width = int(min(wl.P, max(1024, target_wp // wl.N)))
+    small = wl.scaled(width)
+    x = synth.make_params(small, "cpu")
+    xb = x.view(torch.int16).numpy().view(np.uint16) if wl.dtype == "bf16" else x.numpy()
+    grads = synth.make_grads(small, 0, "cpu").numpy() if wl.fused_sgd else None
+    if grads is not None and wl.dtype == "bf16":
+        grads = None
+    w = synth.make_weights(wl, "cpu")
+    wn = w.numpy() if w is not None else None
+    reps = max(1, int(round(target_wp / float(wl.N * width))))
+    oracle.select_peers(wl.sampler_seed, 0, wl.N, wl.S, wl.R)        # loads the library
+    t0 = time.perf_counter()
+    for t in range(reps):
+        idx = oracle.select_peers(wl.sampler_seed, t, wl.N, wl.S, wl.R)
+        oracle.segment_aggregate(xb, idx, wl.S, wl.R, weights=wn, grads=grads, lr=wl.lr, P=wl.P,
+                                 p_begin=0, p_end=width)
+    dt = time.perf_counter() - t0
+    wp = wl.N * width * reps
+    desc = "%d round(s), all %d workers, columns [0,%d) of %d (%d worker-params)" % (
+        reps, wl.N, width, wl.P, wp)
+    return wp / dt, desc, wp, dt
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    oracle.build()
+    per_step = 1.0e8
+    for _ in range(args.warmup):
+        oracle_sample(wl, per_step / 4)
+    total_wp, total_t, desc = 0, 0.0, ""
+    for _ in range(args.steps):
+        v, desc, wp, dt = oracle_sample(wl, per_step)
+        total_wp += wp
+        total_t += dt
+    value = total_wp / total_t
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
+        "data": "synthetic",
+        "config": {"workload": wl.name, "N": wl.N, "P": wl.P, "S": wl.S, "R": wl.R,
+                   "rounds_per_step": "bounded sample: " + desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------ our arm
+def main():
+    args = parse_args()
+    from paper_1908_07782_b200 import synth
+    wl = synth.get_workload(args.workload)
+    if args.impl == "reference":
+        return run_reference(args, wl)
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_1908_07782_b200 as combo
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    combo.load()
+    combo.combo_set_kernel_path(args.path)
+    combo.combo_set_tuning(args.tile, args.stages)
+
+    # every rank: an independent replica of the workload (seed offset by rank)
+    seed = 1000 * rank
+    e = elem_bytes(wl)
+    x0 = synth.make_params(wl, dev, seed=seed)
+    bufs = [x0, torch.empty_like(x0)]
+    weights = synth.make_weights(wl, dev)
+    grads = synth.make_grads(wl, 0, dev, seed=1000 + seed) if wl.fused_sgd else None
+    idx = torch.empty((wl.N, wl.S, wl.R), dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def aggregate(src, dst):
+        if wl.dtype == "bf16":
+            combo.combo_segment_aggregate_bf16(src, dst, weights, idx, wl.N, wl.P, wl.S, wl.R)
+        elif wl.fused_sgd:
+            combo.combo_segment_aggregate_sgd(src, grads, wl.lr, dst, weights, idx, wl.N, wl.P, wl.S, wl.R)
+        else:
+            combo.combo_segment_aggregate(src, dst, weights, idx, wl.N, wl.P, wl.S, wl.R)
+
+    agg_events = []
+
+    def step(record):
+        cur = 0
+        for t in range(wl.rounds):
+            combo.combo_select_peers(wl.sampler_seed + rank, t, wl.N, wl.S, wl.R, idx)
+            if record:
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                aggregate(bufs[cur], bufs[1 - cur])
+                b.record(stream)
+                agg_events.append((a, b))
+            else:
+                aggregate(bufs[cur], bufs[1 - cur])
+            cur = 1 - cur
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 0)):
+        step(False)
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ev0 = torch.cuda.Event(enable_timing=True)
+    ev1 = torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(True)
+    ev1.record(stream)
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if sampler else None
+    kernel_path = combo.combo_last_kernel_path()
+    agg_ms = [a.elapsed_time(b) for a, b in agg_events]
+    combo.combo_device_status()
+
+    # ---- end to end: host buffers, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        nbytes = wl.N * wl.P * e
+        h_in = torch.empty((wl.N, wl.P), dtype=x0.dtype).pin_memory()
+        h_in.copy_(x0)
+        h_out = torch.empty_like(h_in).pin_memory()
+        h_w = weights.cpu() if weights is not None else None
+        h_g = None
+        if grads is not None:
+            h_g = torch.empty((wl.N, wl.P), dtype=torch.float32).pin_memory()
+            h_g.copy_(grads)
+        d_w = torch.empty(wl.N, device=dev) if weights is not None else None
+        e2e_steps = max(1, min(args.steps, 5))
+
+        def e2e_step():
+            combo.combo_round_host(h_in, h_g, wl.lr, h_out, e, h_w, wl.sampler_seed + rank, 0, wl.rounds,
+                                   wl.N, wl.P, wl.S, wl.R, bufs[0], grads, bufs[1], d_w, idx)
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e2e_ms = max(a.elapsed_time(b), 1e3 * (time.perf_counter() - t0) if world == 1 else 0.0)
+        e2e = {"ms": e2e_ms, "steps": e2e_steps,
+               "h2d": nbytes * (2 if h_g is not None else 1) + (4 * wl.N if h_w is not None else 0),
+               "d2h": nbytes}
+
+    # ---- max over ranks
+    if world > 1:
+        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0, max(agg_ms) if agg_ms else 0.0],
+                         device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t[0])
+        if e2e:
+            e2e["ms"] = float(t[1])
+
+    if rank == 0:
+        wp_per_step = wl.N * wl.P * wl.rounds * world
+        value = wp_per_step * args.steps / (ms_total * 1e-3)
+        peak_src = "fallback"
+        peak = FALLBACK_HBM_GBS
+        mp = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(mp):
+            try:
+                peak = float(json.load(open(mp))["hbm_gbs"])
+                peak_src = "measured"
+            except (ValueError, KeyError):
+                pass
+        avg_launch_ms = sum(agg_ms) / len(agg_ms)
+        achieved = algorithmic_bytes_per_launch(wl) / (avg_launch_ms * 1e-3) / 1e9
+        traffic = None
+        if os.path.exists(NCU_TRAFFIC_FILE):
+            try:
+                rec = json.load(open(NCU_TRAFFIC_FILE)).get(wl.name)
+                if rec and rec.get("valid"):
+                    traffic = rec["dram_bytes_per_launch"]
+            except ValueError:
+                pass
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "N": wl.N, "P": wl.P, "S": wl.S, "R": wl.R,
+                       "rounds_per_step": wl.rounds, "weights": "sample counts" if wl.weighted else "equal",
+                       "fused_sgd": wl.fused_sgd, "parallelism": "replicas x%d" % world,
+                       "l2": "inputs larger than L2 (%.2f GB in + out per round)" % (2 * wl.N * wl.P * e / 1e9)
+                       if 2 * wl.N * wl.P * e > 4 * 126e6 else "working set fits L2: warm-L2 number",
+                       "kernel_path": {1: "direct", 2: "staged"}.get(kernel_path, "?")},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                         "kernel": "k_staged" if kernel_path == 2 else "k_direct",
+                         "avg_launch_ms": avg_launch_ms, "min_launch_ms": min(agg_ms),
+                         "algorithmic_bytes_per_launch": algorithmic_bytes_per_launch(wl)},
+            "gpu_launches": 2 * wl.rounds * args.steps,
+            "clocks": clocks,
+        }
+        if e2e:
+            line["e2e"] = {"value": wp_per_step * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": UNIT,
+                           "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                           "ms_per_step": e2e["ms"] / e2e["steps"]}
+        if world == 1 and not args.no_cpu_baseline:
+            del bufs, x0
+            import oracle
+            oracle.build()
+            v, desc, wp, dt = oracle_sample(wl, 8.0e8)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": desc + ", %.1f s" % dt}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

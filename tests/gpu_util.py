@@ -80,9 +80,16 @@ def check_against_oracle(x, out, idx_np, S, R, weights=None, grads=None, lr=0.0,
     got = to_bits(out)
     if x.dtype == torch.bfloat16:
         got64 = bf16_bits_to_f64(got)
-        # storage tolerance: one bf16 unit in the last place of the exact value
-        assert (np.abs(got64 - exact) <= bf16_ulp(exact)).all(), "bf16 result off by more than 1 ulp"
         scale = float(np.abs(bf16_bits_to_f64(xb)).max()) if xb.size else 0.0
+        # The stored value is RNE_bf16 of a binary32 accumulation: half a bf16 ulp from
+        # the rounding plus the binary32 budget d = 1e-6 * max|param| of the accumulate
+        # (which dominates only where providers cancel to a value far below max|param|).
+        # For values of ordinary size this is tighter than the one-ulp contract.
+        d = max(1e-6, (2 * R + 3) * 2.0 ** -24) * scale
+        bound = 0.5 * bf16_ulp(np.abs(exact) + d) + d
+        assert (np.abs(got64 - exact) <= bound).all(), "bf16 result outside half an ulp + fp32 budget"
+        big = np.abs(exact) >= 2.0 ** 9 * d
+        assert (np.abs(got64 - exact)[big] <= bf16_ulp(exact)[big]).all(), "bf16 result off by > 1 ulp"
     else:
         scale = float(np.abs(xb).max()) if xb.size else 0.0
         err = float(np.abs(got.astype(np.float64) - exact).max()) if xb.size else 0.0
