@@ -36,7 +36,7 @@ NCU_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic.json")
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="2", help="1..5 or a workload name (default: 2)")
     ap.add_argument("--impl", default="combo", choices=["combo", "reference"])
@@ -62,9 +62,12 @@ def algorithmic_bytes_per_launch(wl):
 
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """nvidia-smi polled every 50 ms in the background; samples are kept with
+    their wall-clock time so that those inside the timed region can be picked."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
@@ -72,13 +75,21 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def wait_first_sample(self, timeout=5.0):
+        t0 = time.time()
+        while self.proc is not None and time.time() - t0 < timeout:
+            if os.path.getsize(self.tmp.name) > 0:
+                return
+            time.sleep(0.05)
+
+    def stop(self, t_begin: float, t_end: float):
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w_max": None}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -88,28 +99,33 @@ class ClockSampler:
             self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for line in self.tmp.read().splitlines():
-            parts = [p.strip() for p in line.split(",")]
+            parts = [q.strip() for q in line.split(",")]
             if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]),
+                             [q.lower().startswith("active") for q in parts[4:8]]))
             except ValueError:
                 continue
-            for name, val in zip(names, parts[4:8]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
         self.tmp.close()
         os.unlink(self.tmp.name)
-        if sm:
-            # samples under load: the upper half of the observed clocks
-            out["sm_mhz"] = statistics.median(sm)
-            out["sm_max_mhz"] = max(mx)
-            out["samples"] = len(sm)
-        out["reasons"] = sorted(reasons)
+        inside = [r for r in rows if t_begin - 0.06 <= r[0] <= t_end + 0.06]
+        if not inside:           # region shorter than the polling period: nearest samples
+            inside = sorted(rows, key=lambda r: abs(r[0] - 0.5 * (t_begin + t_end)))[:3]
+        if inside:
+            out["sm_mhz"] = statistics.median(r[1] for r in inside)
+            out["sm_max_mhz"] = max(r[2] for r in inside)
+            out["power_w_max"] = max(r[3] for r in inside)
+            out["samples"] = len(inside)
+            reasons = set()
+            for r in inside:
+                for name, on in zip(self.NAMES, r[4]):
+                    if on:
+                        reasons.add(name)
+            out["reasons"] = sorted(reasons)
         return out
 
 
@@ -241,10 +257,13 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(max(args.warmup, 0)):
         step(False)
+    if sampler:
+        sampler.wait_first_sample()
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    t_begin = time.time()
     ev0 = torch.cuda.Event(enable_timing=True)
     ev1 = torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
@@ -253,7 +272,8 @@ def main():
     ev1.record(stream)
     barrier()
     ms_total = ev0.elapsed_time(ev1)
-    clocks = sampler.stop() if sampler else None
+    t_end = time.time()
+    clocks = sampler.stop(t_begin, t_end) if sampler else None
     kernel_path = combo.combo_last_kernel_path()
     agg_ms = [a.elapsed_time(b) for a, b in agg_events]
     combo.combo_device_status()

@@ -66,12 +66,13 @@ inline unsigned round_up(unsigned v, unsigned q) { return (v + q - 1) / q * q; }
 struct StagedPlan {
     bool ok;
     int gb;          // shared-memory read granule in bytes
+    int rt;          // R the kernel is specialised on, or -1
     size_t smem;
     int grid;
 };
 
 StagedPlan plan_staged(AggParams& p, int EB, bool sgd, const DeviceInfo& dev) {
-    StagedPlan plan = {false, 16, 0, 0};
+    StagedPlan plan = {false, 16, -1, 0, 0};
     const int V = 16 / EB;
     const int narr = sgd ? 2 : 1;
     const bool unaligned = (p.pitch % V) != 0;
@@ -80,7 +81,10 @@ StagedPlan plan_staged(AggParams& p, int EB, bool sgd, const DeviceInfo& dev) {
     plan.gb = !unaligned ? 16 : (EB == 4 ? 4 : ((p.pitch % 2 == 0) ? 4 : 2));
     const int Tq = 32 * V;
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
-    const unsigned table = round_up(2u * p.N * ((p.R > 0 ? p.R : 1) * 4u + (p.R + 1) * 4u), 128);
+    // the kernel is specialised on R for 1..4 except on the rarely used granules
+    plan.rt = (p.R >= 1 && p.R <= 4 && (plan.gb == 16 || (EB == 2 && plan.gb == 4))) ? p.R : -1;
+    const int rmax = plan.rt >= 0 ? plan.rt : combo::kStagedMaxR;
+    const unsigned table = round_up(2u * p.N * (unsigned)combo::table_entry_bytes(rmax), 128);
     const long long budget = (long long)dev.smem_optin - header - table - 128;
     auto row_bytes = [&](int T) { return (T + p.halo) * EB + (p.halo ? 16 : 0); };
     auto stage_bytes = [&](int T) { return (long long)round_up((unsigned)(p.N * row_bytes(T) * narr), 128); };
@@ -136,8 +140,9 @@ cudaError_t launch_staged_inst(const AggParams& p, const StagedPlan& plan, cudaS
 
 template <int EB, int GB, bool SGD>
 cudaError_t launch_staged_r(const AggParams& p, const StagedPlan& plan, cudaStream_t st, bool specialise) {
-    if (specialise) {
-        switch (p.R) {
+    if (specialise && plan.rt >= 0) {
+        switch (plan.rt) {
+            case 1: return launch_staged_inst<EB, GB, SGD, 1>(p, plan, st);
             case 2: return launch_staged_inst<EB, GB, SGD, 2>(p, plan, st);
             case 3: return launch_staged_inst<EB, GB, SGD, 3>(p, plan, st);
             case 4: return launch_staged_inst<EB, GB, SGD, 4>(p, plan, st);

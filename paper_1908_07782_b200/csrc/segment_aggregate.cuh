@@ -285,19 +285,79 @@ __device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t& phase, in
     return ok;
 }
 
+// Packed binary32 pairs (one instruction, two IEEE operations, round to nearest).
+__device__ __forceinline__ void mul2(float& d0, float& d1, float c, float x0, float x1) {
+    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%2, %2}; mov.b64 rb, {%3, %4}; mul.rn.f32x2 rd, ra, rb; "
+        "mov.b64 {%0, %1}, rd; }"
+        : "=f"(d0), "=f"(d1)
+        : "f"(c), "f"(x0), "f"(x1));
+}
+__device__ __forceinline__ void fma2(float& d0, float& d1, float c, float x0, float x1) {
+    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%2, %2}; mov.b64 rb, {%3, %4}; mov.b64 rd, {%0, %1}; "
+        "fma.rn.f32x2 rd, ra, rb, rd; mov.b64 {%0, %1}, rd; }"
+        : "+f"(d0), "+f"(d1)
+        : "f"(c), "f"(x0), "f"(x1));
+}
+
+// Coefficient table entry of one (slot, row): cf[RMAX+1] floats, then poff[RMAX+1]
+// ints (shared-memory byte offset of each provider's staged row, phase difference to
+// the output row included), padded to 16 bytes.
+__host__ __device__ constexpr int table_entry_bytes(int rmax) { return ((rmax + 1) * 8 + 15) / 16 * 16; }
+
+template <int RMAX>
+struct RowCtx {
+    float cf[RMAX + 1];
+    int poff[RMAX + 1];
+};
+
+template <int RMAX>
+__device__ __forceinline__ void load_entry(const unsigned char* entry, RowCtx<RMAX>& c) {
+    constexpr int ENT = table_entry_bytes(RMAX);
+    uint32_t raw[ENT / 4];
+#pragma unroll
+    for (int i = 0; i < ENT / 16; ++i) {
+        const uint4 v = reinterpret_cast<const uint4*>(entry)[i];
+        raw[4 * i] = v.x; raw[4 * i + 1] = v.y; raw[4 * i + 2] = v.z; raw[4 * i + 3] = v.w;
+    }
+#pragma unroll
+    for (int r = 0; r <= RMAX; ++r) {
+        c.cf[r] = __uint_as_float(raw[r]);
+        c.poff[r] = (int)raw[RMAX + 1 + r];
+    }
+}
+
+// One output-aligned group: self first, then the peers ascending (Eq. 3, fixed order).
+template <int EB, int GB, int RMAX, bool FIXED_R>
+__device__ __forceinline__ void group_fast(const unsigned char* stage, const RowCtx<RMAX>& c, int R, int goff,
+                                           unsigned char* outp) {
+    constexpr int V = ElemOps<EB>::V;
+    float acc[V], x[V];
+    GroupLoad<EB, GB>::run(stage + c.poff[0] + goff, x);
+#pragma unroll
+    for (int i = 0; i < V; i += 2) mul2(acc[i], acc[i + 1], c.cf[0], x[i], x[i + 1]);
+#pragma unroll
+    for (int r = 1; r <= RMAX; ++r) {
+        if (FIXED_R || r <= R) {
+            GroupLoad<EB, GB>::run(stage + c.poff[r] + goff, x);
+#pragma unroll
+            for (int i = 0; i < V; i += 2) fma2(acc[i], acc[i + 1], c.cf[r], x[i], x[i + 1]);
+        }
+    }
+    ElemOps<EB>::store_vec(outp, acc);
+}
+
 template <int EB, int GB, bool SGD, int RT>
 __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p) {
     constexpr int V = ElemOps<EB>::V;
     constexpr int RMAX = (RT >= 0) ? RT : kStagedMaxR;
+    constexpr int ENT = table_entry_bytes(RMAX);
     extern __shared__ __align__(128) unsigned char smem[];
     StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = p.N, R = (RT >= 0) ? RT : p.R;
     const int stages = p.stages;
     const int narr = SGD ? 2 : 1;
-
-    int32_t* tab_peer = reinterpret_cast<int32_t*>(smem + p.tab_off);           // [2][N][R]
-    float* tab_coef = reinterpret_cast<float*>(tab_peer + 2 * N * (R > 0 ? R : 1));  // [2][N][R+1]
+    unsigned char* tab = smem + p.tab_off;                 // [2][N] entries of ENT bytes
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -312,11 +372,10 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
     if (warp == 0) {
         // ------------------------------------------------------------ producer
         long long n = 0;
-        bool alive = true;
-        for (long long tile = blockIdx.x; tile < p.n_tiles && alive; tile += gridDim.x, ++n) {
+        for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % stages);
             const uint32_t ph = (uint32_t)((n / stages) & 1);
-            if (!mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); alive = false; break; }
+            if (!mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); break; }
             long long cs = tile * p.T - p.halo; if (cs < 0) cs = 0;
             long long ce = (tile + 1) * p.T; if (ce > p.width) ce = p.width;
             unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
@@ -387,44 +446,48 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
     const int CH = GT / 32;          // 32-group chunks per row per tile
     const int n_items = N * CH;
     const int ipw = (n_items + kConsumerWarps - 1) / kConsumerWarps;
+    const int it_begin = cw * ipw;
+    const int it_end = (cw + 1) * ipw < n_items ? (cw + 1) * ipw : n_items;
+    const int row_begin = it_begin / CH, chunk_begin = it_begin - row_begin * CH;
     const uint32_t csync = smem_u32(&hdr->csync);
+    const size_t pitch_bytes = (size_t)p.pitch * EB;
 
     long long n = 0;
     for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
         const int s = (int)(n % stages);
         const uint32_t ph = (uint32_t)((n / stages) & 1);
         if (!mbar_wait(smem_u32(&hdr->full[s]), ph)) { staged_fail(3); return; }
-        const TileMeta m = hdr->meta[s];
+        const long long m_cs = hdr->meta[s].cs, m_ce = hdr->meta[s].ce, m_bnd = hdr->meta[s].bnd;
+        const int m_l0 = hdr->meta[s].l0;
         unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
 
-        if (m.l0 != cached_l0) {
-            // coefficient / peer table for segments l0 and l0+1 (rebuilt at most S times per CTA)
+        if (m_l0 != cached_l0) {
+            // table for segments l0 and l0+1 (rebuilt at most S times per CTA)
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(4); return; }
             for (int q = ctid; q < 2 * N; q += kConsumerThreads) {
                 const int slot = q / N, w = q - slot * N;
-                const int l = m.l0 + slot;
+                const int l = m_l0 + slot;
                 if (l < p.S) {
                     const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
-                    float cf[RMAX + 1];
+                    float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);
+                    int* po = reinterpret_cast<int*>(cf + RMAX + 1);
+                    const int a_w = (int)(((long long)w * p.pitch) & (V - 1));
                     const float dw = p.weights ? p.weights[w] : 1.0f;
                     float den = dw;
-#pragma unroll
-                    for (int r = 0; r < RMAX; ++r)
-                        if (r < R) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+                    for (int r = 0; r < R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
                     cf[0] = __fdiv_rn(dw, den);
-#pragma unroll
-                    for (int r = 0; r < RMAX; ++r)
-                        if (r < R) cf[r + 1] = __fdiv_rn(p.weights ? p.weights[peers[r]] : 1.0f, den);
-                    float* tc = tab_coef + ((size_t)slot * N + w) * (R + 1);
-                    int32_t* tp = tab_peer + ((size_t)slot * N + w) * (R > 0 ? R : 1);
-                    tc[0] = cf[0];
-#pragma unroll
-                    for (int r = 0; r < RMAX; ++r)
-                        if (r < R) { tc[r + 1] = cf[r + 1]; tp[r] = peers[r]; }
+                    po[0] = w * p.row_bytes;
+                    for (int r = 0; r < R; ++r) {
+                        const int k = peers[r];
+                        const int a_k = (int)(((long long)k * p.pitch) & (V - 1));
+                        cf[r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                        po[r + 1] = k * p.row_bytes + (a_k - a_w) * EB;
+                    }
+                    for (int r = R; r < RMAX; ++r) { cf[r + 1] = 0.0f; po[r + 1] = po[0]; }
                 }
             }
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
-            cached_l0 = m.l0;
+            cached_l0 = m_l0;
         }
 
         if (SGD) {
@@ -443,71 +506,57 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(6); return; }
         }
 
-        const bool has_bnd = m.bnd < m.ce;     // a segment boundary lies inside the staged columns
-        const long long g_tile0 = tile * (long long)GT;
+        const bool has_bnd = m_bnd < m_ce;     // a segment boundary lies inside the staged columns
+        const long long t0 = tile * (long long)p.T;            // first shifted column of the tile
+        const bool interior = !has_bnd && (tile > 0 || p.halo == 0) && (t0 + p.T <= p.width);
+        const int tile_goff = (int)(t0 - m_cs) * EB + lane * 16;
 
-        int cur_row = -1;
-        int a_w = 0;
-        float cf[RMAX + 1];
-        int poff[RMAX + 1];
-        const int it_end = (cw + 1) * ipw < n_items ? (cw + 1) * ipw : n_items;
-        int row = (cw * ipw) / CH;
-        int chunk = (cw * ipw) - row * CH;
-        for (int item = cw * ipw; item < it_end; ++item) {
-            if (row != cur_row) {
-                cur_row = row;
-                a_w = (int)(((long long)row * p.pitch) & (V - 1));
-                if (!has_bnd) {
-                    const float* tc = tab_coef + (size_t)row * (R + 1);
-                    const int32_t* tp = tab_peer + (size_t)row * (R > 0 ? R : 1);
-                    cf[0] = tc[0];
-                    poff[0] = row * p.row_bytes;
-#pragma unroll
-                    for (int r = 0; r < RMAX; ++r)
-                        if (r < R) {
-                            const int k = tp[r];
-                            const int a_k = (int)(((long long)k * p.pitch) & (V - 1));
-                            cf[r + 1] = tc[r + 1];
-                            poff[r + 1] = k * p.row_bytes + (a_k - a_w) * EB;
-                        }
+        if (interior) {
+            // every group of the tile is whole and lies in segment l0
+            int row = row_begin, chunk = chunk_begin;
+            RowCtx<RMAX> c;
+            int cur_row = -1;
+            unsigned char* orow = nullptr;
+            for (int item = it_begin; item < it_end; ++item) {
+                if (row != cur_row) {
+                    cur_row = row;
+                    load_entry<RMAX>(tab + (size_t)row * ENT, c);
+                    const int a_w = (int)(((long long)row * p.pitch) & (V - 1));
+                    orow = p.out + (size_t)row * pitch_bytes + (size_t)(t0 - a_w) * EB + lane * 16;
                 }
+                group_fast<EB, GB, RMAX, (RT >= 0)>(stage, c, R, tile_goff + chunk * 512, orow + chunk * 512);
+                if (++chunk == CH) { chunk = 0; ++row; }
             }
-            const long long g = g_tile0 + chunk * 32 + lane;
-            const long long c0 = g * V - a_w;
-            const bool full = (c0 >= 0) && (c0 + V <= p.width);
-            if (full && !has_bnd) {
-                const int goff = (int)(g * V - m.cs) * EB;
-                float acc[V], x[V];
-                GroupLoad<EB, GB>::run(stage + poff[0] + goff, x);
-#pragma unroll
-                for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(cf[0], x[i]);
-#pragma unroll
-                for (int r = 0; r < RMAX; ++r)
-                    if (r < R) {
-                        GroupLoad<EB, GB>::run(stage + poff[r + 1] + goff, x);
-#pragma unroll
-                        for (int i = 0; i < V; ++i) acc[i] = fmaf(cf[r + 1], x[i], acc[i]);
+        } else {
+            // first / last tile of the rows, or a tile holding a segment boundary
+            int row = row_begin, chunk = chunk_begin;
+            for (int item = it_begin; item < it_end; ++item) {
+                const int a_w = (int)(((long long)row * p.pitch) & (V - 1));
+                const long long c0 = t0 + (long long)(chunk * 32 + lane) * V - a_w;
+                const bool whole = (c0 >= 0) && (c0 + V <= p.width);
+                const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
+                if (whole && one_seg) {
+                    RowCtx<RMAX> c;
+                    load_entry<RMAX>(tab + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, c);
+                    group_fast<EB, GB, RMAX, (RT >= 0)>(stage, c, R, tile_goff + chunk * 512,
+                                                        p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB);
+                } else {
+                    const long long lo = c0 < 0 ? 0 : c0;
+                    const long long hi = (c0 + V > p.width) ? p.width : c0 + V;
+                    for (long long c = lo; c < hi; ++c) {
+                        const unsigned char* ent = tab + ((size_t)(c >= m_bnd ? 1 : 0) * N + row) * ENT;
+                        const float* cf = reinterpret_cast<const float*>(ent);
+                        const int* po = reinterpret_cast<const int*>(cf + RMAX + 1);
+                        // element c of provider k sits at poff_k + (c + a_w - cs) * EB
+                        const int eoff = (int)(c + a_w - m_cs) * EB;
+                        float acc = __fmul_rn(cf[0], ElemOps<EB>::load(stage + po[0] + eoff));
+                        for (int r = 1; r <= R; ++r)
+                            acc = fmaf(cf[r], ElemOps<EB>::load(stage + po[r] + eoff), acc);
+                        ElemOps<EB>::store(p.out + (size_t)row * pitch_bytes + (size_t)c * EB, acc);
                     }
-                ElemOps<EB>::store_vec(p.out + ((size_t)row * (size_t)p.pitch + (size_t)c0) * EB, acc);
-            } else {
-                // edge of the row or a tile that holds a segment boundary: element by element
-                const long long lo = c0 < 0 ? 0 : c0;
-                const long long hi = (c0 + V > p.width) ? p.width : c0 + V;
-                for (long long c = lo; c < hi; ++c) {
-                    const int slot = (c >= m.bnd) ? 1 : 0;
-                    const float* tc = tab_coef + ((size_t)slot * N + row) * (R + 1);
-                    const int32_t* tp = tab_peer + ((size_t)slot * N + row) * (R > 0 ? R : 1);
-                    const int eoff = (int)(c - m.cs) * EB;
-                    float acc = __fmul_rn(tc[0], ElemOps<EB>::load(stage + row * p.row_bytes + a_w * EB + eoff));
-                    for (int r = 0; r < R; ++r) {
-                        const int k = tp[r];
-                        const int a_k = (int)(((long long)k * p.pitch) & (V - 1));
-                        acc = fmaf(tc[r + 1], ElemOps<EB>::load(stage + k * p.row_bytes + a_k * EB + eoff), acc);
-                    }
-                    ElemOps<EB>::store(p.out + ((size_t)row * (size_t)p.pitch + (size_t)c) * EB, acc);
                 }
+                if (++chunk == CH) { chunk = 0; ++row; }
             }
-            if (++chunk == CH) { chunk = 0; ++row; }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
