@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 direct gather, 2 staged")
+    ap.add_argument("--P", type=int, default=0, help="override the vector length (scaled-down runs)")
+    ap.add_argument("--N", type=int, default=0, help="override the number of workers")
+    ap.add_argument("--rounds", type=int, default=0, help="override the rounds per step")
     ap.add_argument("--tile", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     return ap.parse_args()
@@ -197,6 +200,10 @@ def main():
     args = parse_args()
     from paper_1908_07782_b200 import synth
     wl = synth.get_workload(args.workload)
+    if args.P or args.N or args.rounds:
+        import dataclasses
+        wl = dataclasses.replace(wl, P=args.P or wl.P, N=args.N or wl.N, rounds=args.rounds or wl.rounds,
+                                 name="%s@N=%d,P=%d" % (wl.name, args.N or wl.N, args.P or wl.P))
     if args.impl == "reference":
         return run_reference(args, wl)
 

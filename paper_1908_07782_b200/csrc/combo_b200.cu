@@ -2,6 +2,7 @@
 // planning, launches).  See include/combo_b200.h for the contract.
 #include "../../include/combo_b200.h"
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdio.h>
@@ -71,58 +72,124 @@ struct StagedPlan {
     int grid;
 };
 
-StagedPlan plan_staged(AggParams& p, int EB, bool sgd, const DeviceInfo& dev) {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+int gcd_int(long long a, long long b) { while (b) { long long t = a % b; a = b; b = t; } return (int)a; }
+
+// Tensor map of row class j of one [N][pitch] array: origin = start of row j rounded down
+// to 16 bytes, x extent up to the last local column, rows m*pitch apart.
+bool encode_class_map(CUtensorMap* map, const unsigned char* base, int EB, int j, int m, int N, long long pitch,
+                      long long width, int box_w) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const long long pitch_bytes = pitch * EB;
+    const long long row0 = (long long)j * pitch_bytes;
+    const long long phase = row0 & 15;
+    const int rows = (N - j + m - 1) / m;
+    cuuint64_t dims[2] = {(cuuint64_t)(phase / EB + width), (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)((long long)m * pitch_bytes)};
+    cuuint32_t box[2] = {(cuuint32_t)box_w, (cuuint32_t)rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, EB == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_UINT16, 2,
+                     const_cast<unsigned char*>(base) + row0 - phase, dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(t_cuda_err, sizeof(t_cuda_err), "cuTensorMapEncodeTiled failed with %d", (int)r);
+        return false;
+    }
+    return true;
+}
+
+StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, const DeviceInfo& dev) {
     StagedPlan plan = {false, 16, -1, 0, 0};
     const int V = 16 / EB;
     const int narr = sgd ? 2 : 1;
-    const bool unaligned = (p.pitch % V) != 0;
     if (p.R > combo::kStagedMaxR) return plan;
-    p.halo = unaligned ? V : 0;
+    const long long pitch_bytes = p.pitch * EB;
+    const int m = 16 / gcd_int(16, pitch_bytes % 16 == 0 ? 16 : pitch_bytes % 16);
+    const bool unaligned = m > 1;
+    if ((p.N + m - 1) / m > 256) return plan;                       // box rows
+    if ((unsigned long long)m * (unsigned long long)pitch_bytes >= (1ull << 40)) return plan;
+    if ((unsigned long long)p.width + V >= (1ull << 32)) return plan;
     plan.gb = !unaligned ? 16 : (EB == 4 ? 4 : ((p.pitch % 2 == 0) ? 4 : 2));
-    const int Tq = 32 * V;
-    const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
     // the kernel is specialised on R for 1..4 except on the rarely used granules
     plan.rt = (p.R >= 1 && p.R <= 4 && (plan.gb == 16 || (EB == 2 && plan.gb == 4))) ? p.R : -1;
     const int rmax = plan.rt >= 0 ? plan.rt : combo::kStagedMaxR;
+    const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
     const unsigned table = round_up(2u * p.N * (unsigned)combo::table_entry_bytes(rmax), 128);
     const long long budget = (long long)dev.smem_optin - header - table - 128;
-    auto row_bytes = [&](int T) { return (T + p.halo) * EB + (p.halo ? 16 : 0); };
-    auto stage_bytes = [&](int T) { return (long long)round_up((unsigned)(p.N * row_bytes(T) * narr), 128); };
-    auto tiles = [&](int T) { return (p.width + (p.halo ? V - 1 : 0) + T - 1) / T; };
-    if ((long long)Tq + p.halo > p.L) return plan;
-    if (2 * stage_bytes(Tq) > budget) return plan;
 
-    int T = 0;
-    if (t_tile > 0) {
-        if (t_tile % Tq != 0 || (long long)t_tile + p.halo > p.L || 2 * stage_bytes(t_tile) > budget) return plan;
-        T = t_tile;
+    // candidate tiles: (T, box_w, nbx)
+    struct Cand { int T, box_w, nbx; };
+    Cand cands[combo::kMaxBoxes + 1];
+    int nc = 0;
+    if (unaligned) {
+        cands[nc++] = {256 - V, 256, 1};
     } else {
-        // largest tile whose stage stays near 64 KB, then the candidate with the least
-        // (waves x tile width), a fixed per-tile cost of 32 columns added
-        const long long target = 64 * 1024;
-        int T_hi = Tq;
-        while (T_hi + Tq <= 4096 && (long long)T_hi + Tq + p.halo <= p.L && stage_bytes(T_hi + Tq) <= target &&
-               2 * stage_bytes(T_hi + Tq) <= budget)
-            T_hi += Tq;
-        double best = 0.0;
-        for (int c = T_hi; c >= Tq; c -= Tq) {
-            const long long nt = tiles(c);
-            const long long waves = (nt + dev.sms - 1) / dev.sms;
-            const double cost = (double)waves * (c + 32);
-            if (T == 0 || cost < best * 0.999) { best = cost; T = c; }
-        }
+        if (EB == 4) cands[nc++] = {128, 128, 1};
+        for (int n = 1; n <= combo::kMaxBoxes; ++n) cands[nc++] = {256 * n, 256, n};
     }
-    int stages = (int)(budget / stage_bytes(T));
+    auto stage_bytes = [&](const Cand& c) { return (long long)narr * c.nbx * p.N * c.box_w * EB; };
+    auto tiles = [&](const Cand& c) { return (p.width + c.T - 1) / c.T; };
+    auto feasible = [&](const Cand& c) {
+        return (long long)c.T <= p.L && 2 * stage_bytes(c) <= budget && narr * c.nbx * m <= 32;
+    };
+    int pick = -1;
+    if (t_tile > 0) {
+        for (int i = 0; i < nc; ++i)
+            if (cands[i].T == t_tile && feasible(cands[i])) pick = i;
+        if (pick < 0) return plan;
+    } else {
+        // among tiles whose stage stays near 64 KB: least (waves x (tile width + a fixed
+        // per-tile cost of 32 columns)); the smallest feasible tile if none is that small
+        double best = 0.0;
+        for (int i = 0; i < nc; ++i) {
+            if (!feasible(cands[i])) continue;
+            if (pick >= 0 && stage_bytes(cands[i]) > 64 * 1024) continue;
+            const long long nt = tiles(cands[i]);
+            const long long waves = (nt + dev.sms - 1) / dev.sms;
+            const double cost = (double)waves * (cands[i].T + 32);
+            if (pick < 0 || cost <= best * 1.001) { best = cost; pick = i; }
+        }
+        if (pick < 0) return plan;
+    }
+    const Cand c = cands[pick];
+    int stages = (int)(budget / stage_bytes(c));
     if (stages > combo::kMaxStages) stages = combo::kMaxStages;
     if (t_stages > 0 && t_stages < stages) stages = t_stages;
     if (stages < 2) return plan;
-    p.T = T;
+    p.T = c.T;
+    p.m = m;
+    p.nbx = c.nbx;
+    p.box_w = c.box_w;
     p.stages = stages;
-    p.row_bytes = row_bytes(T);
-    p.stage_bytes = (unsigned)stage_bytes(T);
+    p.row_bytes = c.box_w * EB;
+    p.stage_bytes = (unsigned)stage_bytes(c);
     p.tab_off = header;
     p.stage_off = header + table;
-    p.n_tiles = tiles(T);
+    p.n_tiles = tiles(c);
+    for (int a = 0; a < narr; ++a)
+        for (int j = 0; j < m && j < p.N; ++j)
+            if (!encode_class_map(&maps.map[a][j], a == 0 ? p.in : p.grads, EB, j, m, p.N, p.pitch, p.width,
+                                  c.box_w))
+                return plan;
     plan.smem = (size_t)p.stage_off + (size_t)stages * p.stage_bytes;
     plan.grid = (int)(p.n_tiles < dev.sms ? p.n_tiles : dev.sms);
     plan.ok = plan.grid > 0;
@@ -130,37 +197,44 @@ StagedPlan plan_staged(AggParams& p, int EB, bool sgd, const DeviceInfo& dev) {
 }
 
 template <int EB, int GB, bool SGD, int RT>
-cudaError_t launch_staged_inst(const AggParams& p, const StagedPlan& plan, cudaStream_t st) {
+cudaError_t launch_staged_inst(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan,
+                               cudaStream_t st) {
     auto kern = combo::k_staged<EB, GB, SGD, RT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem);
     if (e != cudaSuccess) return e;
-    kern<<<plan.grid, combo::kStagedThreads, plan.smem, st>>>(p);
+    kern<<<plan.grid, combo::kStagedThreads, plan.smem, st>>>(p, maps);
     return cudaGetLastError();
 }
 
 template <int EB, int GB, bool SGD>
-cudaError_t launch_staged_r(const AggParams& p, const StagedPlan& plan, cudaStream_t st, bool specialise) {
-    if (specialise && plan.rt >= 0) {
-        switch (plan.rt) {
-            case 1: return launch_staged_inst<EB, GB, SGD, 1>(p, plan, st);
-            case 2: return launch_staged_inst<EB, GB, SGD, 2>(p, plan, st);
-            case 3: return launch_staged_inst<EB, GB, SGD, 3>(p, plan, st);
-            case 4: return launch_staged_inst<EB, GB, SGD, 4>(p, plan, st);
-            default: break;
-        }
+cudaError_t launch_staged_r(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan,
+                            cudaStream_t st) {
+    switch (plan.rt) {
+        case 1: return launch_staged_inst<EB, GB, SGD, 1>(p, maps, plan, st);
+        case 2: return launch_staged_inst<EB, GB, SGD, 2>(p, maps, plan, st);
+        case 3: return launch_staged_inst<EB, GB, SGD, 3>(p, maps, plan, st);
+        case 4: return launch_staged_inst<EB, GB, SGD, 4>(p, maps, plan, st);
+        default: return launch_staged_inst<EB, GB, SGD, -1>(p, maps, plan, st);
     }
-    return launch_staged_inst<EB, GB, SGD, -1>(p, plan, st);
 }
 
-cudaError_t launch_staged(const AggParams& p, const StagedPlan& plan, int EB, bool sgd, cudaStream_t st) {
+template <int EB, int GB, bool SGD>
+cudaError_t launch_staged_generic(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan,
+                                  cudaStream_t st) {
+    return launch_staged_inst<EB, GB, SGD, -1>(p, maps, plan, st);
+}
+
+cudaError_t launch_staged(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan, int EB, bool sgd,
+                          cudaStream_t st) {
     if (EB == 4) {
-        if (plan.gb == 16) return sgd ? launch_staged_r<4, 16, true>(p, plan, st, true)
-                                      : launch_staged_r<4, 16, false>(p, plan, st, true);
-        return sgd ? launch_staged_r<4, 4, true>(p, plan, st, false) : launch_staged_r<4, 4, false>(p, plan, st, false);
+        if (plan.gb == 16) return sgd ? launch_staged_r<4, 16, true>(p, maps, plan, st)
+                                      : launch_staged_r<4, 16, false>(p, maps, plan, st);
+        return sgd ? launch_staged_generic<4, 4, true>(p, maps, plan, st)
+                   : launch_staged_generic<4, 4, false>(p, maps, plan, st);
     }
-    if (plan.gb == 16) return launch_staged_r<2, 16, false>(p, plan, st, true);
-    if (plan.gb == 4) return launch_staged_r<2, 4, false>(p, plan, st, true);
-    return launch_staged_r<2, 2, false>(p, plan, st, false);
+    if (plan.gb == 16) return launch_staged_r<2, 16, false>(p, maps, plan, st);
+    if (plan.gb == 4) return launch_staged_r<2, 4, false>(p, maps, plan, st);
+    return launch_staged_generic<2, 2, false>(p, maps, plan, st);
 }
 
 cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo& dev, cudaStream_t st) {
@@ -209,7 +283,6 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
     p.p_begin = p_begin;
     p.width = width;
     p.L = (P_total + S - 1) / S;
-    p.arr_end_al = (long long)(extent & ~(size_t)15);
     p.N = N; p.S = S; p.R = R;
     p.lr = lr;
     const bool sgd = grads != nullptr;
@@ -218,9 +291,10 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
     bool want_staged = t_force_path != 1;
     if (t_force_path == 0 && (long long)N * width < (1 << 16)) want_staged = false;   // too small to pipeline
     if (want_staged) {
-        StagedPlan plan = plan_staged(p, EB, sgd, *dev);
+        combo::TileMaps maps;
+        StagedPlan plan = plan_staged(p, maps, EB, sgd, *dev);
         if (plan.ok) {
-            cudaError_t e = launch_staged(p, plan, EB, sgd, st);
+            cudaError_t e = launch_staged(p, maps, plan, EB, sgd, st);
             if (e != cudaSuccess) return cuda_fail(e, "staged aggregation launch");
             t_last_path = 2;
             return COMBO_OK;

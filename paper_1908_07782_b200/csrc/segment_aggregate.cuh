@@ -3,25 +3,30 @@
 // Eq. 3 couples workers only at equal column p, and the peer table depends on
 // (worker, segment) alone.  The unit of work is therefore a column tile taken
 // through ALL N rows: the N x T block is brought from HBM into shared memory
-// once (one bulk async copy per row, completion counted on an mbarrier), every
-// worker's output for those columns is formed from it (R+1 shared-memory reads
-// per output element instead of R+1 HBM/L2 reads), and the N x T result goes
-// out with streaming 128-bit stores.  HBM traffic is then the compulsory one:
-// each worker-parameter read once and written once.
+// once by tiled TMA copies (completion counted on an mbarrier), every worker's
+// output for those columns is formed from it (R+1 shared-memory reads per
+// output element instead of R+1 HBM/L2 reads), and the N x T result goes out
+// with streaming stores.  HBM traffic is then the compulsory one: each
+// worker-parameter read once and written once.
 //
 //   k_staged  persistent CTAs, 1 producer warp + 16 consumer warps, a ring of
 //             stages; warp-per-row accumulation in binary32
 //   k_direct  plain gather from global memory (any R, any N, tiny segments);
 //             also the "naive (R+1)-reads" contrast case for profiling
 //
-// Row alignment.  The ABI fixes dense [N][pitch] arrays, so a row starts at
-// byte (w*pitch*e) mod 16 =: phase.  Output vectors are aligned per OUTPUT row
-// (group g of row w covers columns [g*V - a_w, g*V - a_w + V), a_w = phase/e);
-// input rows are staged as the 16-byte aligned superset of the tile and read
-// back at the granule their phase difference allows (16, 4 or 2 bytes).  When
-// phases differ, a tile also loads V columns to the left of its nominal start
-// so that every group lies in exactly one tile.
+// Row alignment.  The ABI fixes dense [N][pitch] arrays, so row k starts at
+// byte phase (k*pitch*e) mod 16.  A tensor map needs a 16-byte aligned base
+// and row stride, so the rows are split into m = 16/gcd(16, pitch*e) classes
+// (k mod m): within a class all rows share one phase and are m*pitch apart, a
+// legal stride.  Each class gets its own tensor map whose origin is the row
+// start rounded DOWN to 16 bytes; its box is V = 16/e columns wider than the
+// tile, so a staged row holds the tile's columns at byte offset phase.
+// When all phases are 0 (m = 1) consumers read and write 128-bit vectors; when
+// they differ, lanes take interleaved 4-byte (or 2-byte) words of the row, so
+// that shared-memory reads stay conflict-free and global stores stay
+// contiguous per warp whatever the phases are.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -36,6 +41,8 @@ constexpr int kConsumerThreads = 32 * kConsumerWarps;
 constexpr int kStagedThreads = 32 + kConsumerThreads;
 constexpr int kMaxStages = 8;
 constexpr int kStagedMaxR = 8;
+constexpr int kMaxClasses = 8;
+constexpr int kMaxBoxes = 8;              // x-boxes per tile
 constexpr uint32_t kWaitCap = 1u << 24;   // polls before a wait is declared dead
 
 struct AggParams {
@@ -49,16 +56,22 @@ struct AggParams {
     long long width;     // local columns
     long long L;         // segment length of the whole vector
     long long n_tiles;
-    long long arr_end_al;  // last valid byte of an input array, rounded down to 16
     int N, S, R;
     float lr;
     int T;               // tile width in elements
-    int halo;            // extra columns loaded left of a tile (0 or V)
+    int m;               // row classes (tensor maps per array)
+    int nbx;             // x-boxes per tile
+    int box_w;           // box width in elements (tile part + phase room)
     int stages;
-    int row_bytes;       // shared-memory bytes per staged row
+    int row_bytes;       // shared-memory bytes per staged row of one box = box_w * e
     unsigned tab_off;    // byte offset of the coefficient table in shared memory
     unsigned stage_off;  // byte offset of stage 0
     unsigned stage_bytes;
+};
+
+// Tensor maps of one launch: [array][class], array 0 = parameters, 1 = gradients.
+struct alignas(64) TileMaps {
+    CUtensorMap map[2][kMaxClasses];
 };
 
 // ---------------------------------------------------------------- small helpers
@@ -101,12 +114,6 @@ template <> struct GroupLoad<4, 16> {
         x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
     }
 };
-template <> struct GroupLoad<4, 4> {
-    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[4]) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) x[i] = reinterpret_cast<const float*>(p)[i];
-    }
-};
 template <> struct GroupLoad<2, 16> {
     __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8]) {
         uint4 v = *reinterpret_cast<const uint4*>(p);
@@ -116,20 +123,62 @@ template <> struct GroupLoad<2, 16> {
         x[6] = bf16_widen(v.w & 0xffffu); x[7] = __uint_as_float(v.w & 0xffff0000u);
     }
 };
+// Narrow granules: the lane owns 16/GB pieces of GB bytes, 32*GB bytes apart
+// (consecutive lanes touch consecutive pieces).  `mask` bit i = piece i is inside the row.
+template <> struct GroupLoad<4, 4> {
+    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[4], unsigned mask = 0xfu) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            x[i] = (mask >> i & 1u) ? *reinterpret_cast<const float*>(p + i * 128) : 0.0f;
+    }
+};
 template <> struct GroupLoad<2, 4> {
-    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8]) {
+    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8], unsigned mask = 0xfu) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            uint32_t v = reinterpret_cast<const uint32_t*>(p)[i];
+            const uint32_t v = (mask >> i & 1u) ? *reinterpret_cast<const uint32_t*>(p + i * 128) : 0u;
             x[2 * i] = bf16_widen(v & 0xffffu);
             x[2 * i + 1] = __uint_as_float(v & 0xffff0000u);
         }
     }
 };
 template <> struct GroupLoad<2, 2> {
-    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8]) {
+    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8], unsigned mask = 0xffu) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = bf16_widen(reinterpret_cast<const uint16_t*>(p)[i]);
+        for (int i = 0; i < 8; ++i)
+            x[i] = (mask >> i & 1u) ? bf16_widen(*reinterpret_cast<const uint16_t*>(p + i * 64)) : 0.0f;
+    }
+};
+
+// Stores of the same pieces.
+template <int EB, int GB> struct GroupStore;
+template <int EB> struct GroupStore<EB, 16> {
+    __device__ static __forceinline__ void run(unsigned char* p, const float (&a)[ElemOps<EB>::V], unsigned) {
+        ElemOps<EB>::store_vec(p, a);
+    }
+};
+template <> struct GroupStore<4, 4> {
+    __device__ static __forceinline__ void run(unsigned char* p, const float (&a)[4], unsigned mask) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (mask >> i & 1u) __stcs(reinterpret_cast<float*>(p + i * 128), a[i]);
+    }
+};
+template <> struct GroupStore<2, 4> {
+    __device__ static __forceinline__ void run(unsigned char* p, const float (&a)[8], unsigned mask) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (mask >> i & 1u)
+                __stcs(reinterpret_cast<unsigned int*>(p + i * 128), pack_bf16x2_rn(a[2 * i], a[2 * i + 1]));
+    }
+};
+template <> struct GroupStore<2, 2> {
+    __device__ static __forceinline__ void run(unsigned char* p, const float (&a)[8], unsigned mask) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (mask >> i & 1u)
+                __stcs(reinterpret_cast<unsigned short*>(p + i * 64),
+                       (unsigned short)(pack_bf16x2_rn(a[i], 0.0f) & 0xffffu));
     }
 };
 
@@ -221,7 +270,7 @@ __global__ void __launch_bounds__(256) k_direct(const AggParams p) {
     }
 }
 
-// ---------------------------------------------------------------- mbarrier / bulk copy (PTX)
+// ---------------------------------------------------------------- mbarrier / TMA (PTX)
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
@@ -250,18 +299,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return false;
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+// Tiled 2-D TMA load of one box (x = element column, y = row of the class) into this CTA's
+// shared memory; completion bytes are counted on `bar`.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-        "l"(src), "r"(bytes), "r"(bar)
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
 
 struct TileMeta {
-    long long cs;    // first local column held in the stage
-    long long ce;    // one past the last
     long long bnd;   // local column where segment l0+1 starts
-    int l0;          // segment of column cs
+    int l0;          // segment of the tile's first column
     int pad;
 };
 
@@ -300,8 +349,8 @@ __device__ __forceinline__ void fma2(float& d0, float& d1, float c, float x0, fl
 }
 
 // Coefficient table entry of one (slot, row): cf[RMAX+1] floats, then poff[RMAX+1]
-// ints (shared-memory byte offset of each provider's staged row, phase difference to
-// the output row included), padded to 16 bytes.
+// ints (shared-memory byte offset of each provider's staged row inside a box block,
+// its phase included), padded to 16 bytes.
 __host__ __device__ constexpr int table_entry_bytes(int rmax) { return ((rmax + 1) * 8 + 15) / 16 * 16; }
 
 template <int RMAX>
@@ -326,31 +375,40 @@ __device__ __forceinline__ void load_entry(const unsigned char* entry, RowCtx<RM
     }
 }
 
-// One output-aligned group: self first, then the peers ascending (Eq. 3, fixed order).
-template <int EB, int GB, int RMAX, bool FIXED_R>
-__device__ __forceinline__ void group_fast(const unsigned char* stage, const RowCtx<RMAX>& c, int R, int goff,
-                                           unsigned char* outp) {
+// One lane's share of an item (512 bytes of an output row): self first, then the
+// peers ascending (Eq. 3, fixed order).
+template <int EB, int GB, int RMAX, bool FIXED_R, bool MASKED>
+__device__ __forceinline__ void item_fast(const unsigned char* stage, const RowCtx<RMAX>& c, int R, int goff,
+                                          unsigned char* outp, unsigned mask) {
     constexpr int V = ElemOps<EB>::V;
     float acc[V], x[V];
-    GroupLoad<EB, GB>::run(stage + c.poff[0] + goff, x);
+    if constexpr (GB == 16) GroupLoad<EB, GB>::run(stage + c.poff[0] + goff, x);
+    else if constexpr (MASKED) GroupLoad<EB, GB>::run(stage + c.poff[0] + goff, x, mask);
+    else GroupLoad<EB, GB>::run(stage + c.poff[0] + goff, x);
 #pragma unroll
     for (int i = 0; i < V; i += 2) mul2(acc[i], acc[i + 1], c.cf[0], x[i], x[i + 1]);
 #pragma unroll
     for (int r = 1; r <= RMAX; ++r) {
         if (FIXED_R || r <= R) {
-            GroupLoad<EB, GB>::run(stage + c.poff[r] + goff, x);
+            if constexpr (GB == 16) GroupLoad<EB, GB>::run(stage + c.poff[r] + goff, x);
+            else if constexpr (MASKED) GroupLoad<EB, GB>::run(stage + c.poff[r] + goff, x, mask);
+            else GroupLoad<EB, GB>::run(stage + c.poff[r] + goff, x);
 #pragma unroll
             for (int i = 0; i < V; i += 2) fma2(acc[i], acc[i + 1], c.cf[r], x[i], x[i + 1]);
         }
     }
-    ElemOps<EB>::store_vec(outp, acc);
+    GroupStore<EB, GB>::run(outp, acc, mask);
 }
 
 template <int EB, int GB, bool SGD, int RT>
-__global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p) {
+__global__ void __launch_bounds__(kStagedThreads, 1)
+k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     constexpr int V = ElemOps<EB>::V;
     constexpr int RMAX = (RT >= 0) ? RT : kStagedMaxR;
     constexpr int ENT = table_entry_bytes(RMAX);
+    constexpr int PIECES = 16 / GB;            // pieces a lane owns per item
+    constexpr int PSTRIDE = 32 * GB;           // bytes between a lane's pieces
+    constexpr int EPP = GB / EB;               // elements per piece
     extern __shared__ __align__(128) unsigned char smem[];
     StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -358,6 +416,7 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
     const int stages = p.stages;
     const int narr = SGD ? 2 : 1;
     unsigned char* tab = smem + p.tab_off;                 // [2][N] entries of ENT bytes
+    const int block_bytes = N * p.row_bytes;               // one x-box of all rows
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -371,59 +430,34 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
+        // lane -> one TMA box per tile: (array a, x-box b, class j)
+        const int per_arr = p.nbx * p.m;
+        const int a = lane / per_arr, rem = lane - a * per_arr;
+        const int b = rem / p.m, j = rem - b * p.m;
+        const bool issuer = lane < narr * per_arr && j < N;
+        int class_base = 0;                                 // staged row index of the class's first row
+        for (int q = 0; q < j; ++q) class_base += (N - q + p.m - 1) / p.m;
+        const CUtensorMap* my_map = &maps.map[issuer ? a : 0][issuer ? j : 0];
+        const uint32_t my_dst_off = (uint32_t)((a * p.nbx + b) * block_bytes + class_base * p.row_bytes);
+        const int tile_cols_per_box = p.T / p.nbx;
         long long n = 0;
         for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % stages);
             const uint32_t ph = (uint32_t)((n / stages) & 1);
             if (!mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); break; }
-            long long cs = tile * p.T - p.halo; if (cs < 0) cs = 0;
-            long long ce = (tile + 1) * p.T; if (ce > p.width) ce = p.width;
-            unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
-            uint32_t my_bytes = 0;
-            for (int k = lane; k < N; k += 32) {
-                const long long b0 = ((long long)k * p.pitch + cs) * EB;
-                const long long b1 = ((long long)k * p.pitch + ce) * EB;
-                const long long A = b0 & ~15LL;
-                long long E = (b1 + 15) & ~15LL;
-                if (E > p.arr_end_al) E = p.arr_end_al;
-                if (E < A) E = A;
-                my_bytes += (uint32_t)(E - A) * narr;
-                if (E < b1) {
-                    // the array ends inside this 16-byte granule: fetch the last elements by hand
-                    for (int a = 0; a < narr; ++a) {
-                        const unsigned char* src = (a == 0 ? p.in : p.grads);
-                        unsigned char* dst = stage + ((size_t)a * N + k) * p.row_bytes;
-                        for (long long b = (E > b0 ? E : b0); b < b1; b += EB) {
-                            if (EB == 4) *reinterpret_cast<uint32_t*>(dst + (b - A)) = *reinterpret_cast<const uint32_t*>(src + b);
-                            else *reinterpret_cast<uint16_t*>(dst + (b - A)) = *reinterpret_cast<const uint16_t*>(src + b);
-                        }
-                    }
-                }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) my_bytes += __shfl_xor_sync(0xffffffffu, my_bytes, o);
-            if (lane == 0) {
-                TileMeta& m = hdr->meta[s];
-                const int l0 = (int)((p.p_begin + cs) / p.L);
-                m.cs = cs; m.ce = ce; m.l0 = l0;
-                m.bnd = (long long)(l0 + 1) * p.L - p.p_begin;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive_expect_tx(smem_u32(&hdr->full[s]), my_bytes);
-            __syncwarp();
+            const long long t0 = tile * (long long)p.T;
             const uint32_t bar = smem_u32(&hdr->full[s]);
-            for (int k = lane; k < N; k += 32) {
-                const long long b0 = ((long long)k * p.pitch + cs) * EB;
-                const long long b1 = ((long long)k * p.pitch + ce) * EB;
-                const long long A = b0 & ~15LL;
-                long long E = (b1 + 15) & ~15LL;
-                if (E > p.arr_end_al) E = p.arr_end_al;
-                if (E > A) {
-                    bulk_g2s(smem_u32(stage + (size_t)k * p.row_bytes), p.in + A, (uint32_t)(E - A), bar);
-                    if (SGD)
-                        bulk_g2s(smem_u32(stage + ((size_t)N + k) * p.row_bytes), p.grads + A, (uint32_t)(E - A), bar);
-                }
+            if (lane == 0) {
+                TileMeta& mt = hdr->meta[s];
+                const int l0 = (int)((p.p_begin + t0) / p.L);
+                mt.l0 = l0;
+                mt.bnd = (long long)(l0 + 1) * p.L - p.p_begin;
+                mbar_arrive_expect_tx(bar, p.stage_bytes);
             }
+            __syncwarp();
+            if (issuer)
+                tma_load_2d(smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) + my_dst_off, my_map,
+                            (int)(t0 + (long long)b * tile_cols_per_box), 0, bar);
         }
         // Leave last: every stage this warp armed must have landed before the CTA's
         // shared memory can be released, even if the consumers gave up.
@@ -442,8 +476,8 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
     const int ctid = tid - 32;
     uint32_t csync_phase = 0;
     int cached_l0 = -1;
-    const int GT = p.T / V;          // groups per tile
-    const int CH = GT / 32;          // 32-group chunks per row per tile
+    const int TB = p.T * EB;                       // payload bytes of a row in a tile
+    const int CH = (TB + 511) / 512;               // 512-byte items per row per tile
     const int n_items = N * CH;
     const int ipw = (n_items + kConsumerWarps - 1) / kConsumerWarps;
     const int it_begin = cw * ipw;
@@ -451,13 +485,15 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
     const int row_begin = it_begin / CH, chunk_begin = it_begin - row_begin * CH;
     const uint32_t csync = smem_u32(&hdr->csync);
     const size_t pitch_bytes = (size_t)p.pitch * EB;
+    const int box_payload = (p.T / p.nbx) * EB;    // tile bytes per row held by one x-box
+    const int box_skip = block_bytes - box_payload;  // extra offset per x-box crossed
 
     long long n = 0;
     for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
         const int s = (int)(n % stages);
         const uint32_t ph = (uint32_t)((n / stages) & 1);
         if (!mbar_wait(smem_u32(&hdr->full[s]), ph)) { staged_fail(3); return; }
-        const long long m_cs = hdr->meta[s].cs, m_ce = hdr->meta[s].ce, m_bnd = hdr->meta[s].bnd;
+        const long long m_bnd = hdr->meta[s].bnd;
         const int m_l0 = hdr->meta[s].l0;
         unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
 
@@ -471,19 +507,21 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
                     const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
                     float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);
                     int* po = reinterpret_cast<int*>(cf + RMAX + 1);
-                    const int a_w = (int)(((long long)w * p.pitch) & (V - 1));
                     const float dw = p.weights ? p.weights[w] : 1.0f;
                     float den = dw;
                     for (int r = 0; r < R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
                     cf[0] = __fdiv_rn(dw, den);
-                    po[0] = w * p.row_bytes;
-                    for (int r = 0; r < R; ++r) {
-                        const int k = peers[r];
-                        const int a_k = (int)(((long long)k * p.pitch) & (V - 1));
-                        cf[r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
-                        po[r + 1] = k * p.row_bytes + (a_k - a_w) * EB;
+                    for (int r = 0; r <= R; ++r) {
+                        const int k = (r == 0) ? w : peers[r - 1];
+                        if (r > 0) cf[r] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                        // staged row of worker k: classes are stored one after another
+                        const int jk = k % p.m;
+                        int base = 0;
+                        for (int q2 = 0; q2 < jk; ++q2) base += (N - q2 + p.m - 1) / p.m;
+                        const int phase = (int)(((long long)k * p.pitch * EB) & 15);
+                        po[r] = (base + k / p.m) * p.row_bytes + phase;
                     }
-                    for (int r = R; r < RMAX; ++r) { cf[r + 1] = 0.0f; po[r + 1] = po[0]; }
+                    for (int r = R + 1; r <= RMAX; ++r) { cf[r] = 0.0f; po[r] = po[0]; }
                 }
             }
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
@@ -492,9 +530,9 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
 
         if (SGD) {
             // local step on the staged tile, in place: x <- fma(-lr, g, x), every row
-            const int nvec = N * p.row_bytes / 16;
+            const int nvec = p.nbx * block_bytes / 16;
             float4* xs = reinterpret_cast<float4*>(stage);
-            const float4* gs = reinterpret_cast<const float4*>(stage + (size_t)N * p.row_bytes);
+            const float4* gs = reinterpret_cast<const float4*>(stage + (size_t)p.nbx * block_bytes);
             const float nlr = -p.lr;
             for (int v = ctid; v < nvec; v += kConsumerThreads) {
                 float4 x = xs[v];
@@ -506,57 +544,76 @@ __global__ void __launch_bounds__(kStagedThreads, 1) k_staged(const AggParams p)
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(6); return; }
         }
 
-        const bool has_bnd = m_bnd < m_ce;     // a segment boundary lies inside the staged columns
-        const long long t0 = tile * (long long)p.T;            // first shifted column of the tile
-        const bool interior = !has_bnd && (tile > 0 || p.halo == 0) && (t0 + p.T <= p.width);
-        const int tile_goff = (int)(t0 - m_cs) * EB + lane * 16;
+        const long long t0 = tile * (long long)p.T;
+        const long long t1 = (t0 + p.T < p.width) ? t0 + p.T : p.width;
+        const bool interior = (m_bnd >= t1) && (t0 + p.T <= p.width);   // one segment, whole tile
 
-        if (interior) {
-            // every group of the tile is whole and lies in segment l0
-            int row = row_begin, chunk = chunk_begin;
-            RowCtx<RMAX> c;
-            int cur_row = -1;
-            unsigned char* orow = nullptr;
-            for (int item = it_begin; item < it_end; ++item) {
+        int row = row_begin, chunk = chunk_begin;
+        RowCtx<RMAX> c;
+        int cur_row = -1;
+        unsigned char* orow = nullptr;
+        for (int item = it_begin; item < it_end; ++item) {
+            const int ib = chunk * 512;                                  // byte offset of the item in the row
+            const int xb = ib / box_payload;                             // x-box holding it
+            const int goff = ib + xb * box_skip + lane * GB;
+            const bool ragged = ib + 512 > TB;                           // item sticks out of the tile row
+            if (interior && (GB == 16 || !ragged)) {
                 if (row != cur_row) {
                     cur_row = row;
                     load_entry<RMAX>(tab + (size_t)row * ENT, c);
-                    const int a_w = (int)(((long long)row * p.pitch) & (V - 1));
-                    orow = p.out + (size_t)row * pitch_bytes + (size_t)(t0 - a_w) * EB + lane * 16;
+                    orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
                 }
-                group_fast<EB, GB, RMAX, (RT >= 0)>(stage, c, R, tile_goff + chunk * 512, orow + chunk * 512);
-                if (++chunk == CH) { chunk = 0; ++row; }
-            }
-        } else {
-            // first / last tile of the rows, or a tile holding a segment boundary
-            int row = row_begin, chunk = chunk_begin;
-            for (int item = it_begin; item < it_end; ++item) {
-                const int a_w = (int)(((long long)row * p.pitch) & (V - 1));
-                const long long c0 = t0 + (long long)(chunk * 32 + lane) * V - a_w;
-                const bool whole = (c0 >= 0) && (c0 + V <= p.width);
-                const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
-                if (whole && one_seg) {
-                    RowCtx<RMAX> c;
-                    load_entry<RMAX>(tab + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, c);
-                    group_fast<EB, GB, RMAX, (RT >= 0)>(stage, c, R, tile_goff + chunk * 512,
-                                                        p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB);
-                } else {
-                    const long long lo = c0 < 0 ? 0 : c0;
-                    const long long hi = (c0 + V > p.width) ? p.width : c0 + V;
-                    for (long long c = lo; c < hi; ++c) {
-                        const unsigned char* ent = tab + ((size_t)(c >= m_bnd ? 1 : 0) * N + row) * ENT;
-                        const float* cf = reinterpret_cast<const float*>(ent);
-                        const int* po = reinterpret_cast<const int*>(cf + RMAX + 1);
-                        // element c of provider k sits at poff_k + (c + a_w - cs) * EB
-                        const int eoff = (int)(c + a_w - m_cs) * EB;
-                        float acc = __fmul_rn(cf[0], ElemOps<EB>::load(stage + po[0] + eoff));
-                        for (int r = 1; r <= R; ++r)
-                            acc = fmaf(cf[r], ElemOps<EB>::load(stage + po[r] + eoff), acc);
-                        ElemOps<EB>::store(p.out + (size_t)row * pitch_bytes + (size_t)c * EB, acc);
+                item_fast<EB, GB, RMAX, (RT >= 0), false>(stage, c, R, goff, orow + ib, 0xffu);
+            } else if (interior) {
+                if (row != cur_row) {
+                    cur_row = row;
+                    load_entry<RMAX>(tab + (size_t)row * ENT, c);
+                    orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
+                }
+                unsigned mask = 0;
+#pragma unroll
+                for (int i = 0; i < PIECES; ++i)
+                    if (ib + lane * GB + i * PSTRIDE < TB) mask |= 1u << i;
+                item_fast<EB, GB, RMAX, (RT >= 0), true>(stage, c, R, goff, orow + ib, mask);
+            } else {
+                // last tile of the rows, or a tile holding a segment boundary: element by element,
+                // except whole 128-bit groups that lie in one segment
+                bool done = false;
+                if (GB == 16) {
+                    const long long c0 = t0 + (ib + lane * 16) / EB;
+                    const bool whole = c0 + V <= p.width;
+                    const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
+                    if (whole && one_seg) {
+                        RowCtx<RMAX> cc;
+                        load_entry<RMAX>(tab + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
+                        item_fast<EB, GB, RMAX, (RT >= 0), false>(
+                            stage, cc, R, goff, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
+                        done = true;
                     }
                 }
-                if (++chunk == CH) { chunk = 0; ++row; }
+                if (!done) {
+#pragma unroll 1
+                    for (int i = 0; i < PIECES; ++i) {
+                        const int pb = ib + lane * GB + i * PSTRIDE;     // byte offset of the piece in the row
+                        if (pb >= TB) continue;
+#pragma unroll 1
+                        for (int e = 0; e < EPP; ++e) {
+                            const long long col = t0 + pb / EB + e;
+                            if (col >= p.width) continue;
+                            const unsigned char* ent = tab + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
+                            const float* cf = reinterpret_cast<const float*>(ent);
+                            const int* po = reinterpret_cast<const int*>(cf + RMAX + 1);
+                            const int eoff = pb + e * EB + (pb / box_payload) * box_skip;
+                            float acc = __fmul_rn(cf[0], ElemOps<EB>::load(stage + po[0] + eoff));
+                            for (int r = 1; r <= R; ++r)
+                                acc = fmaf(cf[r], ElemOps<EB>::load(stage + po[r] + eoff), acc);
+                            ElemOps<EB>::store(p.out + (size_t)row * pitch_bytes + (size_t)col * EB, acc);
+                        }
+                    }
+                }
+                cur_row = -1;
             }
+            if (++chunk == CH) { chunk = 0; ++row; }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));

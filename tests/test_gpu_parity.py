@@ -131,10 +131,11 @@ def test_aggregate_medium_both_kernels(N, P, S, R, dtype, weighted, path):
         check_against_oracle(x, out, idx_np, S, R, weights=weights, grads=grads, lr=0.01)
 
 
-@pytest.mark.parametrize("tile,stages", [(128, 2), (128, 8), (256, 3), (1024, 2), (0, 0)])
+@pytest.mark.parametrize("tile,stages", [(128, 2), (128, 8), (256, 3), (512, 2), (1024, 3), (0, 0)])
 def test_staged_tile_shapes(tile, stages):
-    # many tiles per CTA, ragged last tile, segment boundaries inside tiles
-    N, P, S, R = 16, 1_000_003, 6, 3
+    # many tiles per CTA, several TMA boxes per tile, ragged last tile, segment
+    # boundaries inside tiles
+    N, P, S, R = 16, 1_000_004, 6, 3
     x, grads, counts = _inputs(N, P, torch.float32, 5)
     idx_np = oracle.select_peers(9, 0, N, S, R)
     idx = torch.from_numpy(idx_np).to(DEV)
@@ -143,14 +144,36 @@ def test_staged_tile_shapes(tile, stages):
         out, used = gpu_aggregate(x, idx, S, R, weights=counts, path=combo.PATH_STAGED)
         assert used == combo.PATH_STAGED
         check_against_oracle(x, out, idx_np, S, R, weights=counts)
-        xb = x[:, :600_010].contiguous().to(torch.bfloat16)
-        t16 = tile if tile % 256 == 0 else 0
-        combo.combo_set_tuning(t16, stages)
+        out, used = gpu_aggregate(x, idx, S, R, weights=counts, grads=grads, lr=0.01, path=combo.PATH_STAGED)
+        if tile <= 512:
+            assert used == combo.PATH_STAGED
+        check_against_oracle(x, out, idx_np, S, R, weights=counts, grads=grads, lr=0.01)
+        xb = x[:, :600_016].contiguous().to(torch.bfloat16)
+        combo.combo_set_tuning(tile if tile % 256 == 0 else 0, stages)
         outb, used = gpu_aggregate(xb, idx, S, R, path=combo.PATH_STAGED)
         assert used == combo.PATH_STAGED
         check_against_oracle(xb, outb, idx_np, S, R)
     finally:
         combo.combo_set_tuning(0, 0)
+
+
+@pytest.mark.parametrize("P,dtype", [(1_000_001, torch.float32), (1_000_002, torch.float32),
+                                     (1_000_003, torch.float32), (600_001, torch.bfloat16),
+                                     (600_002, torch.bfloat16), (600_004, torch.bfloat16),
+                                     (600_006, torch.bfloat16)])
+def test_staged_unaligned_rows(P, dtype):
+    # row pitches of every residue: 2, 4 or 8 row classes, 4- and 2-byte granules
+    N, S, R = 13, 5, 4
+    x, grads, counts = _inputs(N, P, dtype, 21)
+    idx_np = oracle.select_peers(4, 1, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    out, used = gpu_aggregate(x, idx, S, R, weights=counts, path=combo.PATH_STAGED)
+    assert used == combo.PATH_STAGED
+    check_against_oracle(x, out, idx_np, S, R, weights=counts)
+    if dtype == torch.float32:
+        out, used = gpu_aggregate(x, idx, S, R, grads=grads, lr=0.01, path=combo.PATH_STAGED)
+        assert used == combo.PATH_STAGED
+        check_against_oracle(x, out, idx_np, S, R, grads=grads, lr=0.01)
 
 
 def test_special_cases_on_device():
