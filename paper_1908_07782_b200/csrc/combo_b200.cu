@@ -134,7 +134,7 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     const int rmax = plan.rt >= 0 ? plan.rt : combo::kStagedMaxR;
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
     const unsigned table = round_up(2u * p.N * (unsigned)combo::table_entry_bytes(rmax), 128);
-    const long long budget = (long long)dev.smem_optin - header - table - 128;
+    const long long budget = (long long)dev.smem_optin - header - table - 256;
 
     // candidate tiles: (T, box_w, nbx)
     struct Cand { int T, box_w, nbx; };
@@ -190,7 +190,8 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
             if (!encode_class_map(&maps.map[a][j], a == 0 ? p.in : p.grads, EB, j, m, p.N, p.pitch, p.width,
                                   c.box_w))
                 return plan;
-    plan.smem = (size_t)p.stage_off + (size_t)stages * p.stage_bytes;
+    // 16 bytes of slack: unmasked reads of a ragged item may run a row phase past the last row
+    plan.smem = (size_t)p.stage_off + (size_t)stages * p.stage_bytes + 16;
     plan.grid = (int)(p.n_tiles < dev.sms ? p.n_tiles : dev.sms);
     plan.ok = plan.grid > 0;
     return plan;

@@ -123,62 +123,101 @@ template <> struct GroupLoad<2, 16> {
         x[6] = bf16_widen(v.w & 0xffffu); x[7] = __uint_as_float(v.w & 0xffff0000u);
     }
 };
-// Narrow granules: the lane owns 16/GB pieces of GB bytes, 32*GB bytes apart
-// (consecutive lanes touch consecutive pieces).  `mask` bit i = piece i is inside the row.
-template <> struct GroupLoad<4, 4> {
-    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[4], unsigned mask = 0xfu) {
+// ---- packed binary32 pairs -----------------------------------------------------
+// Two binary32 values travel in one 64-bit register (low half = first element), the
+// operand form of the f32x2 instructions: one instruction, two IEEE operations.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pair_bits(uint32_t lo, uint32_t hi) { return ((f32x2)hi << 32) | (f32x2)lo; }
+__device__ __forceinline__ f32x2 pair_dup(float c) { return pair_bits(__float_as_uint(c), __float_as_uint(c)); }
+__device__ __forceinline__ float pair_lo(f32x2 v) { return __uint_as_float((uint32_t)v); }
+__device__ __forceinline__ float pair_hi(f32x2 v) { return __uint_as_float((uint32_t)(v >> 32)); }
+__device__ __forceinline__ f32x2 mul2(f32x2 c, f32x2 x) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(c), "l"(x));
+    return d;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 c, f32x2 x, f32x2 acc) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(c), "l"(x));
+    return acc;
+}
+// a 32-bit word holding two bf16 -> the pair of their binary32 values
+__device__ __forceinline__ f32x2 bf16x2_widen(uint32_t w) { return pair_bits(w << 16, w & 0xffff0000u); }
+
+// One lane's share of a 512-byte item as V/2 pairs.  GB = 16: one 128-bit vector at the
+// lane's 16 bytes.  Narrower granules: the lane owns 16/GB pieces of GB bytes, 32*GB
+// bytes apart, so that consecutive lanes touch consecutive pieces whatever the row phase.
+template <int EB, int GB> struct PairLoad;
+template <> struct PairLoad<4, 16> {
+    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[2]) {
+        const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
+        x[0] = v.x; x[1] = v.y;
+    }
+};
+template <> struct PairLoad<2, 16> {
+    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[4]) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p);
+        x[0] = bf16x2_widen(v.x); x[1] = bf16x2_widen(v.y); x[2] = bf16x2_widen(v.z); x[3] = bf16x2_widen(v.w);
+    }
+};
+template <> struct PairLoad<4, 4> {
+    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[2]) {
+        x[0] = pair_bits(*reinterpret_cast<const uint32_t*>(p), *reinterpret_cast<const uint32_t*>(p + 128));
+        x[1] = pair_bits(*reinterpret_cast<const uint32_t*>(p + 256), *reinterpret_cast<const uint32_t*>(p + 384));
+    }
+};
+template <> struct PairLoad<2, 4> {
+    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[4]) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) x[i] = bf16x2_widen(*reinterpret_cast<const uint32_t*>(p + i * 128));
+    }
+};
+template <> struct PairLoad<2, 2> {
+    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[4]) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            x[i] = (mask >> i & 1u) ? *reinterpret_cast<const float*>(p + i * 128) : 0.0f;
-    }
-};
-template <> struct GroupLoad<2, 4> {
-    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8], unsigned mask = 0xfu) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t v = (mask >> i & 1u) ? *reinterpret_cast<const uint32_t*>(p + i * 128) : 0u;
-            x[2 * i] = bf16_widen(v & 0xffffu);
-            x[2 * i + 1] = __uint_as_float(v & 0xffff0000u);
-        }
-    }
-};
-template <> struct GroupLoad<2, 2> {
-    __device__ static __forceinline__ void run(const unsigned char* p, float (&x)[8], unsigned mask = 0xffu) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            x[i] = (mask >> i & 1u) ? bf16_widen(*reinterpret_cast<const uint16_t*>(p + i * 64)) : 0.0f;
+            x[i] = pair_bits((uint32_t)*reinterpret_cast<const uint16_t*>(p + (2 * i) * 64) << 16,
+                             (uint32_t)*reinterpret_cast<const uint16_t*>(p + (2 * i + 1) * 64) << 16);
     }
 };
 
-// Stores of the same pieces.
-template <int EB, int GB> struct GroupStore;
-template <int EB> struct GroupStore<EB, 16> {
-    __device__ static __forceinline__ void run(unsigned char* p, const float (&a)[ElemOps<EB>::V], unsigned) {
-        ElemOps<EB>::store_vec(p, a);
+// Stores of the same pieces; bit i of `mask` = piece i lies inside the row.
+template <int EB, int GB> struct PairStore;
+template <> struct PairStore<4, 16> {
+    __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[2], unsigned) {
+        __stcs(reinterpret_cast<ulonglong2*>(p), make_ulonglong2(a[0], a[1]));
     }
 };
-template <> struct GroupStore<4, 4> {
-    __device__ static __forceinline__ void run(unsigned char* p, const float (&a)[4], unsigned mask) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (mask >> i & 1u) __stcs(reinterpret_cast<float*>(p + i * 128), a[i]);
+template <> struct PairStore<2, 16> {
+    __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[4], unsigned) {
+        __stcs(reinterpret_cast<uint4*>(p),
+               make_uint4(pack_bf16x2_rn(pair_lo(a[0]), pair_hi(a[0])), pack_bf16x2_rn(pair_lo(a[1]), pair_hi(a[1])),
+                          pack_bf16x2_rn(pair_lo(a[2]), pair_hi(a[2])), pack_bf16x2_rn(pair_lo(a[3]), pair_hi(a[3]))));
     }
 };
-template <> struct GroupStore<2, 4> {
-    __device__ static __forceinline__ void run(unsigned char* p, const float (&a)[8], unsigned mask) {
+template <> struct PairStore<4, 4> {
+    __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[2], unsigned mask) {
+        if (mask & 1u) __stcs(reinterpret_cast<float*>(p), pair_lo(a[0]));
+        if (mask & 2u) __stcs(reinterpret_cast<float*>(p + 128), pair_hi(a[0]));
+        if (mask & 4u) __stcs(reinterpret_cast<float*>(p + 256), pair_lo(a[1]));
+        if (mask & 8u) __stcs(reinterpret_cast<float*>(p + 384), pair_hi(a[1]));
+    }
+};
+template <> struct PairStore<2, 4> {
+    __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[4], unsigned mask) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
             if (mask >> i & 1u)
-                __stcs(reinterpret_cast<unsigned int*>(p + i * 128), pack_bf16x2_rn(a[2 * i], a[2 * i + 1]));
+                __stcs(reinterpret_cast<unsigned int*>(p + i * 128), pack_bf16x2_rn(pair_lo(a[i]), pair_hi(a[i])));
     }
 };
-template <> struct GroupStore<2, 2> {
-    __device__ static __forceinline__ void run(unsigned char* p, const float (&a)[8], unsigned mask) {
+template <> struct PairStore<2, 2> {
+    __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[4], unsigned mask) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-            if (mask >> i & 1u)
-                __stcs(reinterpret_cast<unsigned short*>(p + i * 64),
-                       (unsigned short)(pack_bf16x2_rn(a[i], 0.0f) & 0xffffu));
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t w = pack_bf16x2_rn(pair_lo(a[i]), pair_hi(a[i]));
+            if (mask >> (2 * i) & 1u) __stcs(reinterpret_cast<unsigned short*>(p + (2 * i) * 64), (unsigned short)(w & 0xffffu));
+            if (mask >> (2 * i + 1) & 1u) __stcs(reinterpret_cast<unsigned short*>(p + (2 * i + 1) * 64), (unsigned short)(w >> 16));
+        }
     }
 };
 
@@ -334,20 +373,6 @@ __device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t& phase, in
     return ok;
 }
 
-// Packed binary32 pairs (one instruction, two IEEE operations, round to nearest).
-__device__ __forceinline__ void mul2(float& d0, float& d1, float c, float x0, float x1) {
-    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%2, %2}; mov.b64 rb, {%3, %4}; mul.rn.f32x2 rd, ra, rb; "
-        "mov.b64 {%0, %1}, rd; }"
-        : "=f"(d0), "=f"(d1)
-        : "f"(c), "f"(x0), "f"(x1));
-}
-__device__ __forceinline__ void fma2(float& d0, float& d1, float c, float x0, float x1) {
-    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%2, %2}; mov.b64 rb, {%3, %4}; mov.b64 rd, {%0, %1}; "
-        "fma.rn.f32x2 rd, ra, rb, rd; mov.b64 {%0, %1}, rd; }"
-        : "+f"(d0), "+f"(d1)
-        : "f"(c), "f"(x0), "f"(x1));
-}
-
 // Coefficient table entry of one (slot, row): cf[RMAX+1] floats, then poff[RMAX+1]
 // ints (shared-memory byte offset of each provider's staged row inside a box block,
 // its phase included), padded to 16 bytes.
@@ -355,7 +380,7 @@ __host__ __device__ constexpr int table_entry_bytes(int rmax) { return ((rmax + 
 
 template <int RMAX>
 struct RowCtx {
-    float cf[RMAX + 1];
+    f32x2 c2[RMAX + 1];    // coefficient of each provider, duplicated into a pair
     int poff[RMAX + 1];
 };
 
@@ -370,34 +395,32 @@ __device__ __forceinline__ void load_entry(const unsigned char* entry, RowCtx<RM
     }
 #pragma unroll
     for (int r = 0; r <= RMAX; ++r) {
-        c.cf[r] = __uint_as_float(raw[r]);
+        c.c2[r] = pair_bits(raw[r], raw[r]);
         c.poff[r] = (int)raw[RMAX + 1 + r];
     }
 }
 
 // One lane's share of an item (512 bytes of an output row): self first, then the
-// peers ascending (Eq. 3, fixed order).
-template <int EB, int GB, int RMAX, bool FIXED_R, bool MASKED>
+// peers ascending (Eq. 3, fixed order).  Loads are never masked: a piece beyond the
+// row's payload reads bytes that still lie inside the stage (or its 16-byte slack)
+// and its result is dropped by the store mask.
+template <int EB, int GB, int RMAX, bool FIXED_R>
 __device__ __forceinline__ void item_fast(const unsigned char* stage, const RowCtx<RMAX>& c, int R, int goff,
                                           unsigned char* outp, unsigned mask) {
-    constexpr int V = ElemOps<EB>::V;
-    float acc[V], x[V];
-    if constexpr (GB == 16) GroupLoad<EB, GB>::run(stage + c.poff[0] + goff, x);
-    else if constexpr (MASKED) GroupLoad<EB, GB>::run(stage + c.poff[0] + goff, x, mask);
-    else GroupLoad<EB, GB>::run(stage + c.poff[0] + goff, x);
+    constexpr int NP = ElemOps<EB>::V / 2;
+    f32x2 acc[NP], x[NP];
+    PairLoad<EB, GB>::run(stage + c.poff[0] + goff, x);
 #pragma unroll
-    for (int i = 0; i < V; i += 2) mul2(acc[i], acc[i + 1], c.cf[0], x[i], x[i + 1]);
+    for (int i = 0; i < NP; ++i) acc[i] = mul2(c.c2[0], x[i]);
 #pragma unroll
     for (int r = 1; r <= RMAX; ++r) {
         if (FIXED_R || r <= R) {
-            if constexpr (GB == 16) GroupLoad<EB, GB>::run(stage + c.poff[r] + goff, x);
-            else if constexpr (MASKED) GroupLoad<EB, GB>::run(stage + c.poff[r] + goff, x, mask);
-            else GroupLoad<EB, GB>::run(stage + c.poff[r] + goff, x);
+            PairLoad<EB, GB>::run(stage + c.poff[r] + goff, x);
 #pragma unroll
-            for (int i = 0; i < V; i += 2) fma2(acc[i], acc[i + 1], c.cf[r], x[i], x[i + 1]);
+            for (int i = 0; i < NP; ++i) acc[i] = fma2(c.c2[r], x[i], acc[i]);
         }
     }
-    GroupStore<EB, GB>::run(outp, acc, mask);
+    PairStore<EB, GB>::run(outp, acc, mask);
 }
 
 template <int EB, int GB, bool SGD, int RT>
@@ -487,6 +510,8 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     const size_t pitch_bytes = (size_t)p.pitch * EB;
     const int box_payload = (p.T / p.nbx) * EB;    // tile bytes per row held by one x-box
     const int box_skip = block_bytes - box_payload;  // extra offset per x-box crossed
+    // x-box of a byte offset: payloads are powers of two when there are several boxes
+    const int box_shift = (p.nbx > 1) ? (31 - __clz(box_payload)) : 30;
 
     long long n = 0;
     for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
@@ -554,27 +579,22 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         unsigned char* orow = nullptr;
         for (int item = it_begin; item < it_end; ++item) {
             const int ib = chunk * 512;                                  // byte offset of the item in the row
-            const int xb = ib / box_payload;                             // x-box holding it
+            const int xb = ib >> box_shift;                              // x-box holding it
             const int goff = ib + xb * box_skip + lane * GB;
-            const bool ragged = ib + 512 > TB;                           // item sticks out of the tile row
-            if (interior && (GB == 16 || !ragged)) {
+            if (interior) {
                 if (row != cur_row) {
                     cur_row = row;
                     load_entry<RMAX>(tab + (size_t)row * ENT, c);
                     orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
                 }
-                item_fast<EB, GB, RMAX, (RT >= 0), false>(stage, c, R, goff, orow + ib, 0xffu);
-            } else if (interior) {
-                if (row != cur_row) {
-                    cur_row = row;
-                    load_entry<RMAX>(tab + (size_t)row * ENT, c);
-                    orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
-                }
-                unsigned mask = 0;
+                unsigned mask = 0xffu;
+                if (GB != 16 && ib + 512 > TB) {                         // item sticks out of the tile row
+                    mask = 0;
 #pragma unroll
-                for (int i = 0; i < PIECES; ++i)
-                    if (ib + lane * GB + i * PSTRIDE < TB) mask |= 1u << i;
-                item_fast<EB, GB, RMAX, (RT >= 0), true>(stage, c, R, goff, orow + ib, mask);
+                    for (int i = 0; i < PIECES; ++i)
+                        if (ib + lane * GB + i * PSTRIDE < TB) mask |= 1u << i;
+                }
+                item_fast<EB, GB, RMAX, (RT >= 0)>(stage, c, R, goff, orow + ib, mask);
             } else {
                 // last tile of the rows, or a tile holding a segment boundary: element by element,
                 // except whole 128-bit groups that lie in one segment
@@ -586,7 +606,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                     if (whole && one_seg) {
                         RowCtx<RMAX> cc;
                         load_entry<RMAX>(tab + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
-                        item_fast<EB, GB, RMAX, (RT >= 0), false>(
+                        item_fast<EB, GB, RMAX, (RT >= 0)>(
                             stage, cc, R, goff, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
                         done = true;
                     }
@@ -603,7 +623,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                             const unsigned char* ent = tab + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
                             const float* cf = reinterpret_cast<const float*>(ent);
                             const int* po = reinterpret_cast<const int*>(cf + RMAX + 1);
-                            const int eoff = pb + e * EB + (pb / box_payload) * box_skip;
+                            const int eoff = pb + e * EB + (pb >> box_shift) * box_skip;
                             float acc = __fmul_rn(cf[0], ElemOps<EB>::load(stage + po[0] + eoff));
                             for (int r = 1; r <= R; ++r)
                                 acc = fmaf(cf[r], ElemOps<EB>::load(stage + po[r] + eoff), acc);
