@@ -143,7 +143,6 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     if (unaligned) {
         cands[nc++] = {256 - V, 256, 1};
     } else {
-        if (EB == 4) cands[nc++] = {128, 128, 1};
         for (int n = 1; n <= combo::kMaxBoxes; ++n) cands[nc++] = {256 * n, 256, n};
     }
     auto stage_bytes = [&](const Cand& c) { return (long long)narr * c.nbx * p.N * c.box_w * EB; };

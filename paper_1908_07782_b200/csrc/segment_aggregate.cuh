@@ -43,7 +43,8 @@ constexpr int kMaxStages = 8;
 constexpr int kStagedMaxR = 8;
 constexpr int kMaxClasses = 8;
 constexpr int kMaxBoxes = 8;              // x-boxes per tile
-constexpr uint32_t kWaitCap = 1u << 24;   // polls before a wait is declared dead
+constexpr uint32_t kWaitCap = 1u << 23;   // polls before a wait is declared dead
+constexpr uint32_t kWaitHintNs = 1000;    // time a single poll may stay suspended
 
 struct AggParams {
     const unsigned char* in;
@@ -194,20 +195,24 @@ template <> struct PairStore<2, 16> {
                           pack_bf16x2_rn(pair_lo(a[2]), pair_hi(a[2])), pack_bf16x2_rn(pair_lo(a[3]), pair_hi(a[3]))));
     }
 };
+// 32-bit streaming store executed only where `on` is non-zero (predicated, no branch)
+__device__ __forceinline__ void stcs_b32_if(unsigned char* p, uint32_t v, unsigned on) {
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; @q st.global.cs.b32 [%0], %1; }" ::"l"(p), "r"(v), "r"(on)
+                 : "memory");
+}
 template <> struct PairStore<4, 4> {
     __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[2], unsigned mask) {
-        if (mask & 1u) __stcs(reinterpret_cast<float*>(p), pair_lo(a[0]));
-        if (mask & 2u) __stcs(reinterpret_cast<float*>(p + 128), pair_hi(a[0]));
-        if (mask & 4u) __stcs(reinterpret_cast<float*>(p + 256), pair_lo(a[1]));
-        if (mask & 8u) __stcs(reinterpret_cast<float*>(p + 384), pair_hi(a[1]));
+        stcs_b32_if(p, (uint32_t)a[0], mask & 1u);
+        stcs_b32_if(p + 128, (uint32_t)(a[0] >> 32), mask & 2u);
+        stcs_b32_if(p + 256, (uint32_t)a[1], mask & 4u);
+        stcs_b32_if(p + 384, (uint32_t)(a[1] >> 32), mask & 8u);
     }
 };
 template <> struct PairStore<2, 4> {
     __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[4], unsigned mask) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            if (mask >> i & 1u)
-                __stcs(reinterpret_cast<unsigned int*>(p + i * 128), pack_bf16x2_rn(pair_lo(a[i]), pair_hi(a[i])));
+            stcs_b32_if(p + i * 128, pack_bf16x2_rn(pair_lo(a[i]), pair_hi(a[i])), mask & (1u << i));
     }
 };
 template <> struct PairStore<2, 2> {
@@ -329,12 +334,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     for (uint32_t it = 0; it < kWaitCap; ++it) {
         uint32_t ok;
         asm volatile(
-            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
             : "=r"(ok)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(kWaitHintNs)
             : "memory");
         if (ok) return true;
-        if (it > 4096) __nanosleep(64);
     }
     return false;
 }
@@ -373,10 +377,10 @@ __device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t& phase, in
     return ok;
 }
 
-// Coefficient table entry of one (slot, row): cf[RMAX+1] floats, then poff[RMAX+1]
-// ints (shared-memory byte offset of each provider's staged row inside a box block,
-// its phase included), padded to 16 bytes.
-__host__ __device__ constexpr int table_entry_bytes(int rmax) { return ((rmax + 1) * 8 + 15) / 16 * 16; }
+// Coefficient table entry of one (slot, row): c2[RMAX+1] coefficients, each already
+// duplicated into a binary32 pair, then poff[RMAX+1] ints (shared-memory byte offset
+// of each provider's staged row inside a box block, its phase included); padded to 16.
+__host__ __device__ constexpr int table_entry_bytes(int rmax) { return ((rmax + 1) * 12 + 15) / 16 * 16; }
 
 template <int RMAX>
 struct RowCtx {
@@ -395,8 +399,8 @@ __device__ __forceinline__ void load_entry(const unsigned char* entry, RowCtx<RM
     }
 #pragma unroll
     for (int r = 0; r <= RMAX; ++r) {
-        c.c2[r] = pair_bits(raw[r], raw[r]);
-        c.poff[r] = (int)raw[RMAX + 1 + r];
+        c.c2[r] = pair_bits(raw[2 * r], raw[2 * r + 1]);
+        c.poff[r] = (int)raw[2 * (RMAX + 1) + r];
     }
 }
 
@@ -499,19 +503,25 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     const int ctid = tid - 32;
     uint32_t csync_phase = 0;
     int cached_l0 = -1;
-    const int TB = p.T * EB;                       // payload bytes of a row in a tile
-    const int CH = (TB + 511) / 512;               // 512-byte items per row per tile
-    const int n_items = N * CH;
-    const int ipw = (n_items + kConsumerWarps - 1) / kConsumerWarps;
-    const int it_begin = cw * ipw;
-    const int it_end = (cw + 1) * ipw < n_items ? (cw + 1) * ipw : n_items;
-    const int row_begin = it_begin / CH, chunk_begin = it_begin - row_begin * CH;
+    // A unit of consumer work is one row of one x-box: CPB chunks of 512 bytes.
+    constexpr int CPB = (EB == 4) ? 2 : 1;         // boxes are 256 elements wide
+    const int box_payload = (p.T / p.nbx) * EB;    // tile bytes per row held by one x-box
+    const int n_units = N * p.nbx;
+    const int upw = (n_units + kConsumerWarps - 1) / kConsumerWarps;
+    const int u_begin = cw * upw;
+    const int u_end = (cw + 1) * upw < n_units ? (cw + 1) * upw : n_units;
+    const int row_begin = u_begin / p.nbx, xb_begin = u_begin - row_begin * p.nbx;
     const uint32_t csync = smem_u32(&hdr->csync);
     const size_t pitch_bytes = (size_t)p.pitch * EB;
-    const int box_payload = (p.T / p.nbx) * EB;    // tile bytes per row held by one x-box
-    const int box_skip = block_bytes - box_payload;  // extra offset per x-box crossed
-    // x-box of a byte offset: payloads are powers of two when there are several boxes
-    const int box_shift = (p.nbx > 1) ? (31 - __clz(box_payload)) : 30;
+    // store masks of the unit's chunks: bit i = piece i of this lane lies inside the payload
+    unsigned pmask[CPB];
+#pragma unroll
+    for (int ch = 0; ch < CPB; ++ch) {
+        pmask[ch] = 0;
+#pragma unroll
+        for (int i = 0; i < PIECES; ++i)
+            if (ch * 512 + lane * GB + i * PSTRIDE < box_payload) pmask[ch] |= 1u << i;
+    }
 
     long long n = 0;
     for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
@@ -530,15 +540,14 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                 const int l = m_l0 + slot;
                 if (l < p.S) {
                     const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
-                    float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);
-                    int* po = reinterpret_cast<int*>(cf + RMAX + 1);
+                    float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
+                    int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
                     const float dw = p.weights ? p.weights[w] : 1.0f;
                     float den = dw;
                     for (int r = 0; r < R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
-                    cf[0] = __fdiv_rn(dw, den);
                     for (int r = 0; r <= R; ++r) {
                         const int k = (r == 0) ? w : peers[r - 1];
-                        if (r > 0) cf[r] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                        cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
                         // staged row of worker k: classes are stored one after another
                         const int jk = k % p.m;
                         int base = 0;
@@ -546,7 +555,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                         const int phase = (int)(((long long)k * p.pitch * EB) & 15);
                         po[r] = (base + k / p.m) * p.row_bytes + phase;
                     }
-                    for (int r = R + 1; r <= RMAX; ++r) { cf[r] = 0.0f; po[r] = po[0]; }
+                    for (int r = R + 1; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
                 }
             }
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
@@ -573,67 +582,70 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         const long long t1 = (t0 + p.T < p.width) ? t0 + p.T : p.width;
         const bool interior = (m_bnd >= t1) && (t0 + p.T <= p.width);   // one segment, whole tile
 
-        int row = row_begin, chunk = chunk_begin;
-        RowCtx<RMAX> c;
-        int cur_row = -1;
-        unsigned char* orow = nullptr;
-        for (int item = it_begin; item < it_end; ++item) {
-            const int ib = chunk * 512;                                  // byte offset of the item in the row
-            const int xb = ib >> box_shift;                              // x-box holding it
-            const int goff = ib + xb * box_skip + lane * GB;
-            if (interior) {
+        int row = row_begin, xb = xb_begin;
+        if (interior) {
+            // every unit is whole and lies in segment l0: the lean loop
+            RowCtx<RMAX> c;
+            int cur_row = -1;
+            unsigned char* orow = nullptr;
+            for (int u = u_begin; u < u_end; ++u) {
                 if (row != cur_row) {
                     cur_row = row;
                     load_entry<RMAX>(tab + (size_t)row * ENT, c);
                     orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
                 }
-                unsigned mask = 0xffu;
-                if (GB != 16 && ib + 512 > TB) {                         // item sticks out of the tile row
-                    mask = 0;
+                const unsigned char* ubase = stage + xb * block_bytes + lane * GB;
+                unsigned char* uout = orow + xb * box_payload;
 #pragma unroll
-                    for (int i = 0; i < PIECES; ++i)
-                        if (ib + lane * GB + i * PSTRIDE < TB) mask |= 1u << i;
-                }
-                item_fast<EB, GB, RMAX, (RT >= 0)>(stage, c, R, goff, orow + ib, mask);
-            } else {
-                // last tile of the rows, or a tile holding a segment boundary: element by element,
-                // except whole 128-bit groups that lie in one segment
-                bool done = false;
-                if (GB == 16) {
-                    const long long c0 = t0 + (ib + lane * 16) / EB;
-                    const bool whole = c0 + V <= p.width;
-                    const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
-                    if (whole && one_seg) {
-                        RowCtx<RMAX> cc;
-                        load_entry<RMAX>(tab + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
-                        item_fast<EB, GB, RMAX, (RT >= 0)>(
-                            stage, cc, R, goff, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
-                        done = true;
+                for (int ch = 0; ch < CPB; ++ch)
+                    if (GB == 16 || pmask[ch] != 0)
+                        item_fast<EB, GB, RMAX, (RT >= 0)>(ubase + ch * 512, c, R, 0, uout + ch * 512, pmask[ch]);
+                if (++xb == p.nbx) { xb = 0; ++row; }
+            }
+        } else {
+            // last tile of the rows, or a tile holding a segment boundary: element by element,
+            // except whole 128-bit groups that lie in one segment
+            for (int u = u_begin; u < u_end; ++u) {
+#pragma unroll 1
+                for (int ch = 0; ch < CPB; ++ch) {
+                    const int ib = xb * box_payload + ch * 512;          // byte offset of the item in the row
+                    const unsigned char* ubase = stage + xb * block_bytes + ch * 512 + lane * GB;
+                    bool done = false;
+                    if (GB == 16) {
+                        const long long c0 = t0 + (ib + lane * 16) / EB;
+                        const bool whole = c0 + V <= p.width;
+                        const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
+                        if (whole && one_seg) {
+                            RowCtx<RMAX> cc;
+                            load_entry<RMAX>(tab + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
+                            item_fast<EB, GB, RMAX, (RT >= 0)>(
+                                ubase, cc, R, 0, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
+                            done = true;
+                        }
                     }
-                }
-                if (!done) {
+                    if (!done) {
 #pragma unroll 1
-                    for (int i = 0; i < PIECES; ++i) {
-                        const int pb = ib + lane * GB + i * PSTRIDE;     // byte offset of the piece in the row
-                        if (pb >= TB) continue;
+                        for (int i = 0; i < PIECES; ++i) {
+                            const int pin = ch * 512 + lane * GB + i * PSTRIDE;  // byte offset inside the box payload
+                            if (pin >= box_payload) continue;
 #pragma unroll 1
-                        for (int e = 0; e < EPP; ++e) {
-                            const long long col = t0 + pb / EB + e;
-                            if (col >= p.width) continue;
-                            const unsigned char* ent = tab + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
-                            const float* cf = reinterpret_cast<const float*>(ent);
-                            const int* po = reinterpret_cast<const int*>(cf + RMAX + 1);
-                            const int eoff = pb + e * EB + (pb >> box_shift) * box_skip;
-                            float acc = __fmul_rn(cf[0], ElemOps<EB>::load(stage + po[0] + eoff));
-                            for (int r = 1; r <= R; ++r)
-                                acc = fmaf(cf[r], ElemOps<EB>::load(stage + po[r] + eoff), acc);
-                            ElemOps<EB>::store(p.out + (size_t)row * pitch_bytes + (size_t)col * EB, acc);
+                            for (int e = 0; e < EPP; ++e) {
+                                const long long col = t0 + (xb * box_payload + pin) / EB + e;
+                                if (col >= p.width) continue;
+                                const unsigned char* ent = tab + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
+                                const float* cf = reinterpret_cast<const float*>(ent);       // pairs
+                                const int* po = reinterpret_cast<const int*>(cf + 2 * (RMAX + 1));
+                                const unsigned char* eb = stage + xb * block_bytes + pin + e * EB;
+                                float acc = __fmul_rn(cf[0], ElemOps<EB>::load(eb + po[0]));
+                                for (int r = 1; r <= R; ++r)
+                                    acc = fmaf(cf[2 * r], ElemOps<EB>::load(eb + po[r]), acc);
+                                ElemOps<EB>::store(p.out + (size_t)row * pitch_bytes + (size_t)col * EB, acc);
+                            }
                         }
                     }
                 }
-                cur_row = -1;
+                if (++xb == p.nbx) { xb = 0; ++row; }
             }
-            if (++chunk == CH) { chunk = 0; ++row; }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));

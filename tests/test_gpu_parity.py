@@ -131,7 +131,7 @@ def test_aggregate_medium_both_kernels(N, P, S, R, dtype, weighted, path):
         check_against_oracle(x, out, idx_np, S, R, weights=weights, grads=grads, lr=0.01)
 
 
-@pytest.mark.parametrize("tile,stages", [(128, 2), (128, 8), (256, 3), (512, 2), (1024, 3), (0, 0)])
+@pytest.mark.parametrize("tile,stages", [(256, 2), (256, 8), (512, 3), (768, 2), (1024, 3), (0, 0)])
 def test_staged_tile_shapes(tile, stages):
     # many tiles per CTA, several TMA boxes per tile, ragged last tile, segment
     # boundaries inside tiles
@@ -149,7 +149,7 @@ def test_staged_tile_shapes(tile, stages):
             assert used == combo.PATH_STAGED
         check_against_oracle(x, out, idx_np, S, R, weights=counts, grads=grads, lr=0.01)
         xb = x[:, :600_016].contiguous().to(torch.bfloat16)
-        combo.combo_set_tuning(tile if tile % 256 == 0 else 0, stages)
+        combo.combo_set_tuning(tile, stages)
         outb, used = gpu_aggregate(xb, idx, S, R, path=combo.PATH_STAGED)
         assert used == combo.PATH_STAGED
         check_against_oracle(xb, outb, idx_np, S, R)
