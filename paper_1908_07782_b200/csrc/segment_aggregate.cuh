@@ -523,6 +523,40 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             if (ch * 512 + lane * GB + i * PSTRIDE < box_payload) pmask[ch] |= 1u << i;
     }
 
+    // Coefficient / offset table of segments l0 and l0+1, built by all consumer threads.
+    auto build_table = [&](int l0_build) {
+            for (int q = ctid; q < 2 * N; q += kConsumerThreads) {
+        const int slot = q / N, w = q - slot * N;
+        const int l = l0_build + slot;
+        if (l < p.S) {
+            const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
+            float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
+            int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
+            const float dw = p.weights ? p.weights[w] : 1.0f;
+            float den = dw;
+            for (int r = 0; r < R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+            for (int r = 0; r <= R; ++r) {
+                const int k = (r == 0) ? w : peers[r - 1];
+                cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                // staged row of worker k: classes are stored one after another
+                const int jk = k % p.m;
+                int base = 0;
+                for (int q2 = 0; q2 < jk; ++q2) base += (N - q2 + p.m - 1) / p.m;
+                const int phase = (int)(((long long)k * p.pitch * EB) & 15);
+                po[r] = (base + k / p.m) * p.row_bytes + phase;
+            }
+            for (int r = R + 1; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
+        }
+    }
+    };
+    // The first tile's table does not depend on the staged data: build it while the
+    // first TMA loads are in flight.
+    if ((long long)blockIdx.x < p.n_tiles) {
+        cached_l0 = (int)((p.p_begin + (long long)blockIdx.x * p.T) / p.L);
+        build_table(cached_l0);
+        if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(7); return; }
+    }
+
     long long n = 0;
     for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
         const int s = (int)(n % stages);
@@ -535,29 +569,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         if (m_l0 != cached_l0) {
             // table for segments l0 and l0+1 (rebuilt at most S times per CTA)
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(4); return; }
-            for (int q = ctid; q < 2 * N; q += kConsumerThreads) {
-                const int slot = q / N, w = q - slot * N;
-                const int l = m_l0 + slot;
-                if (l < p.S) {
-                    const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
-                    float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
-                    int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
-                    const float dw = p.weights ? p.weights[w] : 1.0f;
-                    float den = dw;
-                    for (int r = 0; r < R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
-                    for (int r = 0; r <= R; ++r) {
-                        const int k = (r == 0) ? w : peers[r - 1];
-                        cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
-                        // staged row of worker k: classes are stored one after another
-                        const int jk = k % p.m;
-                        int base = 0;
-                        for (int q2 = 0; q2 < jk; ++q2) base += (N - q2 + p.m - 1) / p.m;
-                        const int phase = (int)(((long long)k * p.pitch * EB) & 15);
-                        po[r] = (base + k / p.m) * p.row_bytes + phase;
-                    }
-                    for (int r = R + 1; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
-                }
-            }
+            build_table(m_l0);
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
             cached_l0 = m_l0;
         }
