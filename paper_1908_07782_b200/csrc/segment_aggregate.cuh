@@ -147,37 +147,55 @@ __device__ __forceinline__ f32x2 bf16x2_widen(uint32_t w) { return pair_bits(w <
 // One lane's share of a 512-byte item as V/2 pairs.  GB = 16: one 128-bit vector at the
 // lane's 16 bytes.  Narrower granules: the lane owns 16/GB pieces of GB bytes, 32*GB
 // bytes apart, so that consecutive lanes touch consecutive pieces whatever the row phase.
+// Shared-memory loads by 32-bit shared-window address (volatile: they must stay behind
+// the mbarrier wait that publishes the stage).
+template <int OFF> __device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1+%2];" : "=r"(v) : "r"(a), "n"(OFF));
+    return v;
+}
+template <int OFF> __device__ __forceinline__ uint32_t lds16(uint32_t a) {
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1+%2];" : "=h"(v) : "r"(a), "n"(OFF));
+    return (uint32_t)v;
+}
+__device__ __forceinline__ void lds128_pairs(uint32_t a, f32x2& x0, f32x2& x1) {
+    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(x0), "=l"(x1) : "r"(a));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+
 template <int EB, int GB> struct PairLoad;
 template <> struct PairLoad<4, 16> {
-    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[2]) {
-        const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
-        x[0] = v.x; x[1] = v.y;
-    }
+    __device__ static __forceinline__ void run(uint32_t a, f32x2 (&x)[2]) { lds128_pairs(a, x[0], x[1]); }
 };
 template <> struct PairLoad<2, 16> {
-    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[4]) {
-        const uint4 v = *reinterpret_cast<const uint4*>(p);
+    __device__ static __forceinline__ void run(uint32_t a, f32x2 (&x)[4]) {
+        const uint4 v = lds128(a);
         x[0] = bf16x2_widen(v.x); x[1] = bf16x2_widen(v.y); x[2] = bf16x2_widen(v.z); x[3] = bf16x2_widen(v.w);
     }
 };
 template <> struct PairLoad<4, 4> {
-    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[2]) {
-        x[0] = pair_bits(*reinterpret_cast<const uint32_t*>(p), *reinterpret_cast<const uint32_t*>(p + 128));
-        x[1] = pair_bits(*reinterpret_cast<const uint32_t*>(p + 256), *reinterpret_cast<const uint32_t*>(p + 384));
+    __device__ static __forceinline__ void run(uint32_t a, f32x2 (&x)[2]) {
+        x[0] = pair_bits(lds32<0>(a), lds32<128>(a));
+        x[1] = pair_bits(lds32<256>(a), lds32<384>(a));
     }
 };
 template <> struct PairLoad<2, 4> {
-    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[4]) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) x[i] = bf16x2_widen(*reinterpret_cast<const uint32_t*>(p + i * 128));
+    __device__ static __forceinline__ void run(uint32_t a, f32x2 (&x)[4]) {
+        x[0] = bf16x2_widen(lds32<0>(a)); x[1] = bf16x2_widen(lds32<128>(a));
+        x[2] = bf16x2_widen(lds32<256>(a)); x[3] = bf16x2_widen(lds32<384>(a));
     }
 };
 template <> struct PairLoad<2, 2> {
-    __device__ static __forceinline__ void run(const unsigned char* p, f32x2 (&x)[4]) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            x[i] = pair_bits((uint32_t)*reinterpret_cast<const uint16_t*>(p + (2 * i) * 64) << 16,
-                             (uint32_t)*reinterpret_cast<const uint16_t*>(p + (2 * i + 1) * 64) << 16);
+    __device__ static __forceinline__ void run(uint32_t a, f32x2 (&x)[4]) {
+        x[0] = pair_bits(lds16<0>(a) << 16, lds16<64>(a) << 16);
+        x[1] = pair_bits(lds16<128>(a) << 16, lds16<192>(a) << 16);
+        x[2] = pair_bits(lds16<256>(a) << 16, lds16<320>(a) << 16);
+        x[3] = pair_bits(lds16<384>(a) << 16, lds16<448>(a) << 16);
     }
 };
 
@@ -329,10 +347,22 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
                  "r"(bytes)
                  : "memory");
 }
-// Bounded wait: false when the phase did not complete within kWaitCap polls.
+// Bounded wait: false when the phase did not complete within kWaitCap polls.  The first
+// polls return as soon as the hardware allows (hand-offs between producer and consumers
+// are latency critical); later ones let the warp stay suspended for up to kWaitHintNs.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+#pragma unroll 1
+    for (uint32_t it = 0; it < 32; ++it) {
+        asm volatile(
+            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+#pragma unroll 1
     for (uint32_t it = 0; it < kWaitCap; ++it) {
-        uint32_t ok;
         asm volatile(
             "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
             : "=r"(ok)
@@ -409,17 +439,17 @@ __device__ __forceinline__ void load_entry(const unsigned char* entry, RowCtx<RM
 // row's payload reads bytes that still lie inside the stage (or its 16-byte slack)
 // and its result is dropped by the store mask.
 template <int EB, int GB, int RMAX, bool FIXED_R>
-__device__ __forceinline__ void item_fast(const unsigned char* stage, const RowCtx<RMAX>& c, int R, int goff,
-                                          unsigned char* outp, unsigned mask) {
+__device__ __forceinline__ void item_fast(uint32_t base, const RowCtx<RMAX>& c, int R, unsigned char* outp,
+                                          unsigned mask) {
     constexpr int NP = ElemOps<EB>::V / 2;
     f32x2 acc[NP], x[NP];
-    PairLoad<EB, GB>::run(stage + c.poff[0] + goff, x);
+    PairLoad<EB, GB>::run(base + c.poff[0], x);
 #pragma unroll
     for (int i = 0; i < NP; ++i) acc[i] = mul2(c.c2[0], x[i]);
 #pragma unroll
     for (int r = 1; r <= RMAX; ++r) {
         if (FIXED_R || r <= R) {
-            PairLoad<EB, GB>::run(stage + c.poff[r] + goff, x);
+            PairLoad<EB, GB>::run(base + c.poff[r], x);
 #pragma unroll
             for (int i = 0; i < NP; ++i) acc[i] = fma2(c.c2[r], x[i], acc[i]);
         }
@@ -465,6 +495,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         int class_base = 0;                                 // staged row index of the class's first row
         for (int q = 0; q < j; ++q) class_base += (N - q + p.m - 1) / p.m;
         const CUtensorMap* my_map = &maps.map[issuer ? a : 0][issuer ? j : 0];
+        if (issuer) asm volatile("prefetch.tensormap [%0];" ::"l"(my_map) : "memory");
         const uint32_t my_dst_off = (uint32_t)((a * p.nbx + b) * block_bytes + class_base * p.row_bytes);
         const int tile_cols_per_box = p.T / p.nbx;
         long long n = 0;
@@ -565,6 +596,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         const long long m_bnd = hdr->meta[s].bnd;
         const int m_l0 = hdr->meta[s].l0;
         unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
+        const uint32_t stage_s = smem_u32(stage);
 
         if (m_l0 != cached_l0) {
             // table for segments l0 and l0+1 (rebuilt at most S times per CTA)
@@ -606,12 +638,12 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                     load_entry<RMAX>(tab + (size_t)row * ENT, c);
                     orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
                 }
-                const unsigned char* ubase = stage + xb * block_bytes + lane * GB;
+                const uint32_t ubase = stage_s + xb * block_bytes + lane * GB;
                 unsigned char* uout = orow + xb * box_payload;
 #pragma unroll
                 for (int ch = 0; ch < CPB; ++ch)
-                    if (GB == 16 || pmask[ch] != 0)
-                        item_fast<EB, GB, RMAX, (RT >= 0)>(ubase + ch * 512, c, R, 0, uout + ch * 512, pmask[ch]);
+                    if (GB == 16 || ch * 512 < box_payload)
+                        item_fast<EB, GB, RMAX, (RT >= 0)>(ubase + ch * 512, c, R, uout + ch * 512, pmask[ch]);
                 if (++xb == p.nbx) { xb = 0; ++row; }
             }
         } else {
@@ -621,7 +653,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
 #pragma unroll 1
                 for (int ch = 0; ch < CPB; ++ch) {
                     const int ib = xb * box_payload + ch * 512;          // byte offset of the item in the row
-                    const unsigned char* ubase = stage + xb * block_bytes + ch * 512 + lane * GB;
+                    const uint32_t ubase = stage_s + xb * block_bytes + ch * 512 + lane * GB;
                     bool done = false;
                     if (GB == 16) {
                         const long long c0 = t0 + (ib + lane * 16) / EB;
@@ -631,7 +663,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                             RowCtx<RMAX> cc;
                             load_entry<RMAX>(tab + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
                             item_fast<EB, GB, RMAX, (RT >= 0)>(
-                                ubase, cc, R, 0, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
+                                ubase, cc, R, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
                             done = true;
                         }
                     }
