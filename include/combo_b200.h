@@ -156,6 +156,12 @@ combo_status combo_validate_idx(const int32_t* idx, int N, int S, int R, void* s
  * d_grads if h_grads != NULL) [N][P] of elem_bytes each, d_weights float[N]
  * (if h_weights != NULL), d_idx int32[N*S*R].  h_idx_out, if not NULL,
  * receives the peer table of the last round.  rounds >= 1.
+ * Columns are independent in Eq. 3, so the call cuts the vector into column
+ * chunks and overlaps the copy-in of one chunk, all rounds of the previous
+ * one and the copy-out of the one before on three streams (two of them, and
+ * a few events, are created by the first call on a device and kept).  Not
+ * reentrant per device.  After the call d_in and d_out hold intermediate
+ * rounds, not a defined result.
  */
 combo_status combo_round_host(const void* h_params_in, const void* h_grads, float lr,
                               void* h_params_out, int elem_bytes, const float* h_weights,

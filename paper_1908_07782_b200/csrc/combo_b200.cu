@@ -311,6 +311,37 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
     return COMBO_OK;
 }
 
+// Streams and events of the host-memory entry point, created on its first call on a device.
+constexpr int kPipeChunks = 16;
+struct HostPipe {
+    bool ready;
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev_start, ev_end, ev_in[kPipeChunks], ev_done[kPipeChunks];
+};
+HostPipe g_pipe[64];
+
+combo_status host_pipe(HostPipe** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return COMBO_ERR_UNSUPPORTED;
+    HostPipe& h = g_pipe[dev];
+    if (!h.ready) {
+        if ((e = cudaStreamCreateWithFlags(&h.s_in, cudaStreamNonBlocking)) != cudaSuccess ||
+            (e = cudaStreamCreateWithFlags(&h.s_out, cudaStreamNonBlocking)) != cudaSuccess ||
+            (e = cudaEventCreateWithFlags(&h.ev_start, cudaEventDisableTiming)) != cudaSuccess ||
+            (e = cudaEventCreateWithFlags(&h.ev_end, cudaEventDisableTiming)) != cudaSuccess)
+            return cuda_fail(e, "creating the copy streams");
+        for (int i = 0; i < kPipeChunks; ++i)
+            if ((e = cudaEventCreateWithFlags(&h.ev_in[i], cudaEventDisableTiming)) != cudaSuccess ||
+                (e = cudaEventCreateWithFlags(&h.ev_done[i], cudaEventDisableTiming)) != cudaSuccess)
+                return cuda_fail(e, "creating the chunk events");
+        h.ready = true;
+    }
+    *out = &h;
+    return COMBO_OK;
+}
+
 combo_status select_peers_impl(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* idx_out,
                                cudaStream_t st) {
     if (N < 1 || N > COMBO_MAX_WORKERS || S < 1 || S > COMBO_MAX_SEGMENTS || R < 0 || R > N - 1)
@@ -397,33 +428,73 @@ combo_status combo_round_host(const void* h_params_in, const void* h_grads, floa
     if (h_weights && !d_weights) return COMBO_ERR_INVALID_ARG;
     if (elem_bytes != 4 && elem_bytes != 2) return COMBO_ERR_INVALID_ARG;
     if (N < 1 || P < 1 || R < 0 || rounds < 1 || (R > 0 && !d_idx)) return COMBO_ERR_INVALID_ARG;
+    DeviceInfo* dev = nullptr;
+    combo_status rc = device_info(&dev);
+    if (rc != COMBO_OK) return rc;
+    HostPipe* hp = nullptr;
+    rc = host_pipe(&hp);
+    if (rc != COMBO_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t bytes = (size_t)N * (size_t)P * (size_t)elem_bytes;
+    const size_t EB = (size_t)elem_bytes;
+    const size_t pitch_bytes = (size_t)P * EB;
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(d_in, h_params_in, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-        return cuda_fail(e, "copy params to device");
-    if (h_grads && (e = cudaMemcpyAsync(d_grads, h_grads, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-        return cuda_fail(e, "copy grads to device");
     if (h_weights &&
         (e = cudaMemcpyAsync(d_weights, h_weights, sizeof(float) * (size_t)N, cudaMemcpyHostToDevice, st)) !=
             cudaSuccess)
         return cuda_fail(e, "copy weights to device");
-    void* cur = d_in;
-    void* nxt = d_out;
-    for (int t = 0; t < rounds; ++t) {
-        combo_status rc = select_peers_impl(seed, round + (uint32_t)t, N, S, R, d_idx, st);
-        if (rc != COMBO_OK) return rc;
-        rc = aggregate_cols(cur, d_grads, lr, nxt, elem_bytes, h_weights ? d_weights : nullptr, d_idx, N, P, S, R,
-                            0, P, P, stream);
-        if (rc != COMBO_OK) return rc;
-        void* sw = cur; cur = nxt; nxt = sw;
+
+    // Eq. 3 couples workers only at equal column, in every round: a column chunk can run
+    // through ALL rounds on its own.  Chunks are therefore pipelined over three streams:
+    // chunk c+1 is copied in and chunk c-1 copied out while chunk c is aggregated.
+    const size_t total = (size_t)N * pitch_bytes;
+    int K = (int)((total + (64u << 20) - 1) / (64u << 20));
+    if (K > kPipeChunks) K = kPipeChunks;
+    if (K < 1) K = 1;
+    int64_t cw = ((P + K - 1) / K + 63) / 64 * 64;        // chunk width, 16-byte aligned starts
+    if ((e = cudaEventRecord(hp->ev_start, st)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    if ((e = cudaStreamWaitEvent(hp->s_in, hp->ev_start, 0)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(hp->s_out, hp->ev_start, 0)) != cudaSuccess)
+        return cuda_fail(e, "cudaStreamWaitEvent");
+    for (int c = 0; c < K; ++c) {
+        const int64_t p0 = (int64_t)c * cw;
+        if (p0 >= P) break;
+        const int64_t w = (p0 + cw <= P) ? cw : P - p0;
+        const size_t off = (size_t)p0 * EB;
+        if ((e = cudaMemcpy2DAsync(static_cast<char*>(d_in) + off, pitch_bytes,
+                                   static_cast<const char*>(h_params_in) + off, pitch_bytes, (size_t)w * EB,
+                                   (size_t)N, cudaMemcpyHostToDevice, hp->s_in)) != cudaSuccess)
+            return cuda_fail(e, "copy params to device");
+        if (h_grads && (e = cudaMemcpy2DAsync(static_cast<char*>(d_grads) + off, pitch_bytes,
+                                              static_cast<const char*>(h_grads) + off, pitch_bytes, (size_t)w * EB,
+                                              (size_t)N, cudaMemcpyHostToDevice, hp->s_in)) != cudaSuccess)
+            return cuda_fail(e, "copy grads to device");
+        if ((e = cudaEventRecord(hp->ev_in[c], hp->s_in)) != cudaSuccess ||
+            (e = cudaStreamWaitEvent(st, hp->ev_in[c], 0)) != cudaSuccess)
+            return cuda_fail(e, "chunk hand-over to the compute stream");
+        char* cur = static_cast<char*>(d_in) + off;
+        char* nxt = static_cast<char*>(d_out) + off;
+        for (int t = 0; t < rounds; ++t) {
+            rc = select_peers_impl(seed, round + (uint32_t)t, N, S, R, d_idx, st);
+            if (rc != COMBO_OK) return rc;
+            rc = aggregate_cols(cur, d_grads ? static_cast<char*>(d_grads) + off : nullptr, lr, nxt, elem_bytes,
+                                h_weights ? d_weights : nullptr, d_idx, N, P, S, R, p0, w, P, stream);
+            if (rc != COMBO_OK) return rc;
+            char* sw = cur; cur = nxt; nxt = sw;
+        }
+        if ((e = cudaEventRecord(hp->ev_done[c], st)) != cudaSuccess ||
+            (e = cudaStreamWaitEvent(hp->s_out, hp->ev_done[c], 0)) != cudaSuccess)
+            return cuda_fail(e, "chunk hand-over to the copy-out stream");
+        if ((e = cudaMemcpy2DAsync(static_cast<char*>(h_params_out) + off, pitch_bytes, cur, pitch_bytes,
+                                   (size_t)w * EB, (size_t)N, cudaMemcpyDeviceToHost, hp->s_out)) != cudaSuccess)
+            return cuda_fail(e, "copy result to host");
     }
-    if ((e = cudaMemcpyAsync(h_params_out, cur, bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-        return cuda_fail(e, "copy result to host");
     if (h_idx_out && R > 0 &&
         (e = cudaMemcpyAsync(h_idx_out, d_idx, sizeof(int32_t) * (size_t)N * S * R, cudaMemcpyDeviceToHost, st)) !=
             cudaSuccess)
         return cuda_fail(e, "copy idx to host");
+    if ((e = cudaEventRecord(hp->ev_end, hp->s_out)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(st, hp->ev_end, 0)) != cudaSuccess)
+        return cuda_fail(e, "join of the copy-out stream");
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
     return COMBO_OK;
 }

@@ -36,7 +36,10 @@ namespace combo {
 // device status word: 0, or the code of the first bounded wait that gave up
 __device__ int g_dev_status;
 
-constexpr int kConsumerWarps = 16;
+#ifndef COMBO_CONSUMER_WARPS
+#define COMBO_CONSUMER_WARPS 16
+#endif
+constexpr int kConsumerWarps = COMBO_CONSUMER_WARPS;
 constexpr int kConsumerThreads = 32 * kConsumerWarps;
 constexpr int kStagedThreads = 32 + kConsumerThreads;
 constexpr int kMaxStages = 8;

@@ -268,3 +268,44 @@ def test_round_from_host_memory():
         cur = oracle.segment_aggregate_ordered_f32(cur, idx_t, S, R, weights=hw.numpy())
     assert (hidx.numpy() == idx_t).all()
     assert (hout.numpy().view(np.uint32) == cur.view(np.uint32)).all()
+
+
+@pytest.mark.parametrize("P,fused", [(9_000_004, False), (9_000_001, False), (4_500_000, True)])
+def test_round_from_host_memory_in_chunks(P, fused):
+    # large enough for several column chunks to be in flight; the result must equal the
+    # same rounds run on device-resident buffers, bit for bit
+    N, S, R, rounds = 8, 5, 3, 3
+    g = torch.Generator().manual_seed(2)
+    hx = torch.empty(N, P).pin_memory()
+    hx.copy_(torch.randn(N, P, generator=g) * 0.05)
+    hg = None
+    if fused:
+        hg = torch.empty(N, P).pin_memory()
+        hg.copy_(torch.randn(N, P, generator=g) * 1e-3)
+    hw = torch.randint(500, 1501, (N,), generator=g).float()
+    hout = torch.empty_like(hx).pin_memory()
+    d_in = torch.empty(N, P, device=DEV)
+    d_out = torch.empty(N, P, device=DEV)
+    d_g = torch.empty(N, P, device=DEV) if fused else None
+    d_w = torch.empty(N, device=DEV)
+    d_idx = torch.empty((N, S, R), dtype=torch.int32, device=DEV)
+    combo.combo_round_host(hx, hg, 0.01, hout, 4, hw, 5, 0, rounds, N, P, S, R, d_in, d_g, d_out, d_w, d_idx)
+    cur = hx.to(DEV)
+    nxt = torch.empty_like(cur)
+    gd = hg.to(DEV) if fused else None
+    wd = hw.to(DEV)
+    for t in range(rounds):
+        combo.combo_select_peers(5, t, N, S, R, d_idx)
+        if fused:
+            combo.combo_segment_aggregate_sgd(cur, gd, 0.01, nxt, wd, d_idx, N, P, S, R)
+        else:
+            combo.combo_segment_aggregate(cur, nxt, wd, d_idx, N, P, S, R)
+        cur, nxt = nxt, cur
+    torch.cuda.synchronize()
+    assert torch.equal(hout.to(DEV), cur)
+    # and one sampled slab against the oracle, first round only
+    idx0 = oracle.select_peers(5, 0, N, S, R)
+    a, b = P // 2 - 100, P // 2 + 100
+    combo.combo_round_host(hx, hg, 0.01, hout, 4, hw, 5, 0, 1, N, P, S, R, d_in, d_g, d_out, d_w, d_idx)
+    check_against_oracle(hx[:, a:b].contiguous(), hout[:, a:b].contiguous(), idx0, S, R, weights=hw,
+                         grads=hg[:, a:b].contiguous() if fused else None, lr=0.01, P=P, p_begin=a)
