@@ -176,6 +176,24 @@ def test_staged_unaligned_rows(P, dtype):
         check_against_oracle(x, out, idx_np, S, R, grads=grads, lr=0.01)
 
 
+@pytest.mark.parametrize("N,P,S,R,dtype", [
+    (3, 100_001, 2, 2, torch.bfloat16),     # more row classes (8) than workers
+    (2, 100_003, 3, 1, torch.float32),      # two workers, one peer
+    (5, 65_537, 1, 4, torch.float32),       # S = 1 (plain gossip), R = n-1
+    (6, 70_000, 7, 5, torch.bfloat16),      # R without a specialised kernel
+    (200, 3_000, 4, 3, torch.float32),      # many workers, short rows (segments shorter than a tile)
+    (130, 40_000, 2, 2, torch.bfloat16),    # more than 128 workers
+])
+def test_staged_odd_shapes(N, P, S, R, dtype):
+    x, grads, counts = _inputs(N, P, dtype, 77)
+    idx_np = oracle.select_peers(2, 5, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    out, used = gpu_aggregate(x, idx, S, R, weights=counts, path=combo.PATH_STAGED)
+    check_against_oracle(x, out, idx_np, S, R, weights=counts)
+    out2, _ = gpu_aggregate(x, idx, S, R, weights=counts, path=combo.PATH_DIRECT)
+    assert torch.equal(out, out2)                 # both kernels follow the same fixed order
+
+
 def test_special_cases_on_device():
     N, P, S = 6, 100_000, 4
     x, _, counts = _inputs(N, P, torch.float32, 3)
