@@ -67,6 +67,9 @@ def _load():
         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_int, ctypes.c_int64,
         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int,
         ctypes.c_int, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
+    lib.oracle_divergence.restype = ctypes.c_int
+    lib.oracle_divergence.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+                                      ctypes.c_int, ctypes.c_int64, ctypes.c_void_p]
     _lib = lib
     return lib
 
@@ -174,3 +177,27 @@ def segment_aggregate_ordered_f32(x, idx, S, R, weights=None, grads=None, lr=0.0
     if rc != 0:
         raise ValueError("oracle_segment_aggregate_ordered_f32: invalid arguments")
     return out
+
+
+def divergence(models, weights=None, mean_of=None) -> np.ndarray:
+    """Eq. 7: rho_i = || models_i - weighted mean over the rows of mean_of || (binary64,
+    Euclidean norm).  ``mean_of`` defaults to ``models``.  Arrays are float32 or uint16
+    (bf16) [N][P]."""
+    lib = _load()
+    elem = 4 if models.dtype == np.float32 else 2
+    mptr, P = _slab(models, elem)
+    N = models.shape[0]
+    sptr = None
+    if mean_of is not None:
+        sptr, P2 = _slab(mean_of, elem)
+        if P2 != P or mean_of.shape[0] != N:
+            raise ValueError("mean_of shape mismatch")
+    wptr = None
+    if weights is not None:
+        weights = np.ascontiguousarray(weights, dtype=np.float32)
+        wptr = weights.ctypes.data
+    rho = np.zeros(N, dtype=np.float64)
+    rc = lib.oracle_divergence(mptr, sptr, elem, wptr, N, P, rho.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle_divergence: invalid arguments")
+    return rho

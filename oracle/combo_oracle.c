@@ -21,6 +21,10 @@
  *                                when S*R <= n-1), uniformity of the shuffle.
  *                                Its exact tables are PARITY UNPINNED by the
  *                                paper, which names no generator.
+ *   oracle_divergence            exact rational brute force of Eq. 7 on tiny
+ *                                inputs, two-worker closed form, identical
+ *                                models (zero), R = n-1 (zero, as the paper
+ *                                states), scaling and translation laws
  *   oracle_segment_aggregate_*   exact rational brute force of Eq. 3 on tiny
  *                                inputs, hand-worked dyadic example, R = 0,
  *                                R = n-1 (all-reduce / FedAvg mean), S = 1,
@@ -261,5 +265,37 @@ int oracle_segment_aggregate_ordered_f32(const void *in, const void *grads, floa
         }
     }
     free(coef);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* Aggregation divergence (Section 4.3, Definition 2, Eq. 7):          */
+/*   rho_i = || W_{t,i} - W_t ||                                       */
+/* W_{t,i}: the model worker i holds (row i of `models`); W_t: the     */
+/* aggregation of ALL workers, the FedAvg result                       */
+/*   W_t = sum_j |D_j| W_j / sum_j |D_j|                               */
+/* taken over the rows of `mean_of` (the models the round started      */
+/* from; the same array as `models` when mean_of == NULL).  Reading:   */
+/* the norm is the Euclidean one.  Binary64 throughout.                */
+/* models, mean_of: [N][P] dense, elem 4 = binary32, 2 = bf16.         */
+/* ------------------------------------------------------------------ */
+int oracle_divergence(const void *models, const void *mean_of, int elem, const float *weights,
+                      int N, int64_t P, double *rho) {
+    if (N < 1 || P < 1 || (elem != 4 && elem != 2)) return 1;
+    if (!mean_of) mean_of = models;
+    double den = 0.0;
+    for (int j = 0; j < N; ++j) den += weights ? (double)weights[j] : 1.0;
+    for (int i = 0; i < N; ++i) rho[i] = 0.0;
+    for (int64_t p = 0; p < P; ++p) {
+        double num = 0.0;
+        for (int j = 0; j < N; ++j)
+            num += (weights ? (double)weights[j] : 1.0) * load_x(mean_of, elem, (size_t)j * (size_t)P + (size_t)p);
+        double mean = num / den;
+        for (int i = 0; i < N; ++i) {
+            double d = load_x(models, elem, (size_t)i * (size_t)P + (size_t)p) - mean;
+            rho[i] += d * d;
+        }
+    }
+    for (int i = 0; i < N; ++i) rho[i] = sqrt(rho[i]);
     return 0;
 }
