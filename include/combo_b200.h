@@ -26,6 +26,7 @@
 #ifndef COMBO_B200_H
 #define COMBO_B200_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -168,6 +169,29 @@ combo_status combo_round_host(const void* h_params_in, const void* h_grads, floa
                               uint64_t seed, uint32_t round, int rounds, int N, int64_t P, int S,
                               int R, void* d_in, void* d_grads, void* d_out, float* d_weights,
                               int32_t* d_idx, int32_t* h_idx_out, void* stream);
+
+/*
+ * Aggregation divergence -- Section 4.3, Definition 2 (Eq. 7): for every
+ * worker i, rho_i = || W_{t,i} - W_t || (Euclidean norm), where W_{t,i} is row
+ * i of `models` (the worker's aggregation result) and W_t is the aggregation
+ * of ALL workers, the FedAvg result sum_j |D_j| W_j / sum_j |D_j|, taken over
+ * the rows of `mean_of` (the models the round started from).  mean_of == NULL
+ * or == models measures the models against their own weighted mean.  With
+ * R = N-1 every rho_i is zero up to rounding, as the paper states.
+ *
+ * models, mean_of: [N][P] dense, elem_bytes 4 (float) or 2 (bfloat16), read
+ * only.  rho_out: device double[N].  scratch: device memory of at least
+ * combo_divergence_scratch_bytes(N) bytes, 8-byte aligned, used for per-CTA
+ * partial sums (no need to clear it; contents are undefined afterwards).
+ * Arithmetic: column means and deviations in binary32 (weights normalised
+ * first, rows in ascending order), squares summed in binary64; relative error
+ * of rho about 1e-6 for models that differ by more than 1e-3 of their size.
+ * Two launches on `stream`, no synchronisation.
+ */
+size_t combo_divergence_scratch_bytes(int N);
+combo_status combo_aggregation_divergence(const void* models, const void* mean_of, int elem_bytes,
+                                          const float* weights, int N, int64_t P, double* rho_out,
+                                          void* scratch, size_t scratch_bytes, void* stream);
 
 /*
  * Reads and clears the device status word that kernels set when one of their

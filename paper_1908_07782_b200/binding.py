@@ -49,6 +49,7 @@ def load():
         "combo_validate_idx": [vp, i32, i32, i32, vp, vp],
         "combo_round_host": [vp, vp, f32, vp, i32, vp, u64, u32, i32, i32, i64, i32, i32, vp, vp, vp,
                              vp, vp, vp, vp],
+        "combo_aggregation_divergence": [vp, vp, i32, vp, i32, i64, vp, vp, ctypes.c_size_t, vp],
         "combo_device_status": [],
         "combo_last_kernel_path": [],
         "combo_version": [],
@@ -57,6 +58,8 @@ def load():
         fn = getattr(lib, name)
         fn.argtypes = args
         fn.restype = ctypes.c_int
+    lib.combo_divergence_scratch_bytes.argtypes = [i32]
+    lib.combo_divergence_scratch_bytes.restype = ctypes.c_size_t
     lib.combo_set_kernel_path.argtypes = [i32]
     lib.combo_set_kernel_path.restype = None
     lib.combo_set_tuning.argtypes = [i32, i32]
@@ -143,6 +146,21 @@ def combo_round_host(h_params_in, h_grads, lr, h_params_out, elem_bytes, h_weigh
                                    _ptr(d_grads), _ptr(d_out), _ptr(d_weights), _ptr(d_idx),
                                    _ptr(h_idx_out), _stream(stream)), "combo_round_host")
     return h_params_out
+
+
+def combo_divergence_scratch_bytes(N: int) -> int:
+    return int(load().combo_divergence_scratch_bytes(N))
+
+
+def combo_aggregation_divergence(models, mean_of, elem_bytes, weights, N, P, rho_out, scratch, stream=None):
+    """Eq. 7 for all workers: rho_out (float64 [N], device) = distance of each row of
+    ``models`` from the weighted mean over the rows of ``mean_of`` (or of ``models``).
+    ``scratch`` is a device tensor of at least combo_divergence_scratch_bytes(N) bytes."""
+    _check(load().combo_aggregation_divergence(_ptr(models), _ptr(mean_of), elem_bytes, _ptr(weights), N, P,
+                                               _ptr(rho_out), _ptr(scratch),
+                                               scratch.numel() * scratch.element_size(), _stream(stream)),
+           "combo_aggregation_divergence")
+    return rho_out
 
 
 def combo_device_status():

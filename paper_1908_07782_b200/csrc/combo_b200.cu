@@ -9,6 +9,7 @@
 #include <string.h>
 
 #include "segment_aggregate.cuh"
+#include "divergence.cuh"
 #include "select_peers.cuh"
 
 namespace {
@@ -311,6 +312,102 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
     return COMBO_OK;
 }
 
+// ---------------------------------------------------------------- aggregation divergence
+// Blocks whose partial sums the scratch must hold: the staged kernel launches at most one
+// CTA per SM, the fallback at most four.
+inline long long divergence_max_blocks(const DeviceInfo& dev) { return (long long)dev.sms * 4; }
+
+combo_status divergence_impl(const void* models, const void* mean_of, int EB, const float* weights, int N,
+                             long long P, double* rho_out, double* scratch, size_t scratch_bytes, void* stream) {
+    if (EB != 4 && EB != 2) return COMBO_ERR_INVALID_ARG;
+    if (N < 1 || N > COMBO_MAX_WORKERS || P < 1 || !models || !rho_out || !scratch) return COMBO_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(models) & (EB - 1)) || (mean_of && (reinterpret_cast<uintptr_t>(mean_of) & (EB - 1))))
+        return COMBO_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 7) || (reinterpret_cast<uintptr_t>(rho_out) & 7)) return COMBO_ERR_INVALID_ARG;
+    if ((unsigned long long)P > (1ull << 40) / (unsigned)N) return COMBO_ERR_INVALID_ARG;
+    DeviceInfo* dev = nullptr;
+    combo_status rc = device_info(&dev);
+    if (rc != COMBO_OK) return rc;
+    if (scratch_bytes < (size_t)divergence_max_blocks(*dev) * (size_t)N * sizeof(double)) return COMBO_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool two = mean_of != nullptr && mean_of != models;
+
+    combo::DivParams p;
+    memset(&p, 0, sizeof(p));
+    p.models = static_cast<const unsigned char*>(models);
+    p.src = static_cast<const unsigned char*>(two ? mean_of : models);
+    p.weights = weights;
+    p.partial = scratch;
+    p.pitch = P;
+    p.width = P;
+    p.N = N;
+    p.narr = two ? 2 : 1;
+
+    int nblocks = 0;
+    // staged path: 16-byte aligned rows, at most 256 workers, two stages must fit
+    const long long pitch_bytes = P * EB;
+    const bool aligned = (pitch_bytes % 16) == 0 && aligned16(models) && aligned16(p.src);
+    if (t_force_path != 1 && aligned && N <= combo::kDivMaxStagedN && (long long)N * P >= (1 << 16) &&
+        (unsigned long long)P + 256 < (1ull << 31)) {
+        const int V = 16 / EB;
+        const int G = combo::kConsumerThreads / (combo::kDivTile / V);
+        p.row_bytes = combo::kDivTile * EB;
+        const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
+        p.coef_off = header;
+        p.part_off = p.coef_off + round_up((unsigned)N * 4u, 128);
+        p.mean_off = p.part_off + (unsigned)G * combo::kDivTile * 4u;
+        p.stage_off = p.mean_off + combo::kDivTile * 4u;
+        p.stage_bytes = (unsigned)(p.narr * N * p.row_bytes);
+        const long long budget = (long long)dev->smem_optin - p.stage_off - 256;
+        const int fit = (int)(budget / p.stage_bytes);
+        int stages = (int)((112 * 1024) / p.stage_bytes);
+        if (stages < 2) stages = 2;
+        if (stages > combo::kMaxStages) stages = combo::kMaxStages;
+        if (stages > fit) stages = fit;
+        combo::TileMaps maps;
+        if (stages >= 2 &&
+            encode_class_map(&maps.map[0][0], p.models, EB, 0, 1, N, P, P, combo::kDivTile) &&
+            (!two || encode_class_map(&maps.map[1][0], p.src, EB, 0, 1, N, P, P, combo::kDivTile))) {
+            p.stages = stages;
+            p.n_tiles = (P + combo::kDivTile - 1) / combo::kDivTile;
+            nblocks = (int)(p.n_tiles < dev->sms ? p.n_tiles : dev->sms);
+            const size_t smem = (size_t)p.stage_off + (size_t)stages * p.stage_bytes;
+            cudaError_t e;
+            if (EB == 4) {
+                e = cudaFuncSetAttribute(combo::k_divergence_staged<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                if (e == cudaSuccess) combo::k_divergence_staged<4><<<nblocks, combo::kStagedThreads, smem, st>>>(p, maps);
+            } else {
+                e = cudaFuncSetAttribute(combo::k_divergence_staged<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                if (e == cudaSuccess) combo::k_divergence_staged<2><<<nblocks, combo::kStagedThreads, smem, st>>>(p, maps);
+            }
+            if (e == cudaSuccess) e = cudaGetLastError();
+            if (e != cudaSuccess) return cuda_fail(e, "divergence launch");
+            t_last_path = 2;
+        }
+    }
+    if (nblocks == 0) {
+        const long long n_blk = (P + 255) / 256;
+        const long long cap = divergence_max_blocks(*dev);
+        nblocks = (int)(n_blk < cap ? n_blk : cap);
+        const size_t smem = (size_t)N * 12 + 16;
+        cudaError_t e = cudaSuccess;
+        if (EB == 4) {
+            if (smem > 48 * 1024) e = cudaFuncSetAttribute(combo::k_divergence_direct<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e == cudaSuccess) combo::k_divergence_direct<4><<<nblocks, 256, smem, st>>>(p);
+        } else {
+            if (smem > 48 * 1024) e = cudaFuncSetAttribute(combo::k_divergence_direct<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e == cudaSuccess) combo::k_divergence_direct<2><<<nblocks, 256, smem, st>>>(p);
+        }
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e, "divergence launch");
+        t_last_path = 1;
+    }
+    combo::k_divergence_finish<<<(N + 127) / 128, 128, 0, st>>>(scratch, nblocks, N, rho_out);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "divergence finish launch");
+    return COMBO_OK;
+}
+
 // Streams and events of the host-memory entry point, created on its first call on a device.
 constexpr int kPipeChunks = 16;
 struct HostPipe {
@@ -497,6 +594,19 @@ combo_status combo_round_host(const void* h_params_in, const void* h_grads, floa
         return cuda_fail(e, "join of the copy-out stream");
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
     return COMBO_OK;
+}
+
+size_t combo_divergence_scratch_bytes(int N) {
+    DeviceInfo* dev = nullptr;
+    if (N < 1 || N > COMBO_MAX_WORKERS || device_info(&dev) != COMBO_OK) return 0;
+    return (size_t)divergence_max_blocks(*dev) * (size_t)N * sizeof(double);
+}
+
+combo_status combo_aggregation_divergence(const void* models, const void* mean_of, int elem_bytes,
+                                          const float* weights, int N, int64_t P, double* rho_out, void* scratch,
+                                          size_t scratch_bytes, void* stream) {
+    return divergence_impl(models, mean_of, elem_bytes, weights, N, P, rho_out, static_cast<double*>(scratch),
+                           scratch_bytes, stream);
 }
 
 combo_status combo_device_status(void) {
