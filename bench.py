@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="2", help="1..5 or a workload name (default: 2)")
     ap.add_argument("--impl", default="combo", choices=["combo", "reference"])
+    ap.add_argument("--op", default="round", choices=["round", "divergence"],
+                    help="round: the synchronization round (default); divergence: the Eq. 7 diagnostic alone")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 direct gather, 2 staged")
@@ -195,6 +197,60 @@ def run_reference(args, wl):
     return 0
 
 
+# ------------------------------------------------------------------ divergence diagnostic (extra line)
+def run_divergence(args, wl):
+    """Times combo_aggregation_divergence (Eq. 7) on the workload's vectors: aggregated
+    models against the mean of the models the round started from (two arrays read)."""
+    import torch
+
+    import paper_1908_07782_b200 as combo
+    from paper_1908_07782_b200 import synth
+
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    e = elem_bytes(wl)
+    x = synth.make_params(wl, dev)
+    out = torch.empty_like(x)
+    weights = synth.make_weights(wl, dev)
+    idx = torch.empty((wl.N, wl.S, wl.R), dtype=torch.int32, device=dev)
+    combo.combo_select_peers(wl.sampler_seed, 0, wl.N, wl.S, wl.R, idx)
+    if wl.dtype == "bf16":
+        combo.combo_segment_aggregate_bf16(x, out, weights, idx, wl.N, wl.P, wl.S, wl.R)
+    else:
+        combo.combo_segment_aggregate(x, out, weights, idx, wl.N, wl.P, wl.S, wl.R)
+    rho = torch.empty(wl.N, dtype=torch.float64, device=dev)
+    scratch = torch.empty(combo.combo_divergence_scratch_bytes(wl.N) // 8, dtype=torch.float64, device=dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(args.warmup, 3)):
+        combo.combo_aggregation_divergence(out, x, e, weights, wl.N, wl.P, rho, scratch)
+    torch.cuda.synchronize()
+    a = torch.cuda.Event(enable_timing=True)
+    b = torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(args.steps):
+        combo.combo_aggregation_divergence(out, x, e, weights, wl.N, wl.P, rho, scratch)
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    alg = 2 * wl.N * wl.P * e
+    peak, src = FALLBACK_HBM_GBS, "fallback"
+    mp = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(mp):
+        peak, src = float(json.load(open(mp))["hbm_gbs"]), "measured"
+    ach = alg / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "worker_params_measured_per_s", "op": "aggregation_divergence", "value": wl.N * wl.P / (ms * 1e-3),
+        "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "N": wl.N, "P": wl.P, "arrays_read": 2,
+                   "kernel_path": {1: "direct", 2: "staged"}.get(combo.combo_last_kernel_path(), "?")},
+        "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                     "traffic": None, "peak_source": src, "kernel": "k_divergence_staged + k_divergence_finish",
+                     "algorithmic_bytes_per_launch": alg},
+        "gpu_launches": 2 * args.steps, "rho_mean": float(rho.mean())}))
+    return 0
+
+
 # ------------------------------------------------------------------ our arm
 def main():
     args = parse_args()
@@ -206,6 +262,8 @@ def main():
                                  name="%s@N=%d,P=%d" % (wl.name, args.N or wl.N, args.P or wl.P))
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.op == "divergence":
+        return run_divergence(args, wl)
 
     import torch
     import torch.distributed as dist
