@@ -41,12 +41,14 @@ enum {
     COMBO_ERR_ALIAS = 2,          /* input and output ranges overlap             */
     COMBO_ERR_UNSUPPORTED = 3,    /* current device is not compute capability 10.x */
     COMBO_ERR_CUDA = 4,           /* a CUDA runtime call failed; see combo_last_cuda_error */
-    COMBO_ERR_DEVICE_TIMEOUT = 5  /* a bounded wait inside a kernel ran out      */
+    COMBO_ERR_DEVICE_TIMEOUT = 5, /* a bounded wait inside a kernel ran out      */
+    COMBO_ERR_TOO_LARGE = 6       /* beyond the fixed limit of a no-allocation entry point */
 };
 
 /* Limits of this build. */
 #define COMBO_MAX_WORKERS 8192    /* N */
 #define COMBO_MAX_SEGMENTS 65536  /* S */
+#define COMBO_NOALLOC_MAX_WORKERS 128   /* N of combo_aggregation_divergence_noalloc */
 
 /*
  * Peer selection -- Section 4.1, step (2) "Segments Pulling": every worker
@@ -192,6 +194,35 @@ size_t combo_divergence_scratch_bytes(int N);
 combo_status combo_aggregation_divergence(const void* models, const void* mean_of, int elem_bytes,
                                           const float* weights, int N, int64_t P, double* rho_out,
                                           void* scratch, size_t scratch_bytes, void* stream);
+
+/*
+ * combo_aggregation_divergence for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of the call above,
+ * same arithmetic, same result.)
+ *
+ * Who needs it: code that runs where cudaMalloc is not an option -- inside a
+ * region being captured into a CUDA graph or between other work that must not
+ * synchronise the device (cudaMalloc and cudaFree may do both), in a process
+ * whose memory pool is owned and fully handed out by another component, or
+ * in a host language binding that cannot create device buffers at all.  Such
+ * a caller still passes its inputs and the output, but no scratch: the
+ * partial sums go to a fixed array inside the library, 1 MiB that every GPU
+ * loading the library holds until the process exits.
+ *
+ * Limits and rules:
+ *  - N <= COMBO_NOALLOC_MAX_WORKERS (128); more returns COMBO_ERR_TOO_LARGE
+ *    and combo_last_cuda_error() says so.  P is not limited.
+ *  - The first call on each device looks the array's device address up
+ *    (cudaGetSymbolAddress, with that device current) and keeps it; make that
+ *    first call outside any stream capture.  No call allocates or frees.
+ *  - All calls on a device share the one array and it keeps whatever the last
+ *    call left.  Nothing has to be cleared, because every partial sum is
+ *    written before it is read; but two calls that overlap on the GPU (other
+ *    streams, other host threads) race on it -- serialise them on one stream.
+ */
+combo_status combo_aggregation_divergence_noalloc(const void* models, const void* mean_of,
+                                                  int elem_bytes, const float* weights, int N,
+                                                  int64_t P, double* rho_out, void* stream);
 
 /*
  * Reads and clears the device status word that kernels set when one of their

@@ -50,6 +50,7 @@ def load():
         "combo_round_host": [vp, vp, f32, vp, i32, vp, u64, u32, i32, i32, i64, i32, i32, vp, vp, vp,
                              vp, vp, vp, vp],
         "combo_aggregation_divergence": [vp, vp, i32, vp, i32, i64, vp, vp, ctypes.c_size_t, vp],
+        "combo_aggregation_divergence_noalloc": [vp, vp, i32, vp, i32, i64, vp, vp],
         "combo_device_status": [],
         "combo_last_kernel_path": [],
         "combo_version": [],
@@ -160,6 +161,17 @@ def combo_aggregation_divergence(models, mean_of, elem_bytes, weights, N, P, rho
                                                _ptr(rho_out), _ptr(scratch),
                                                scratch.numel() * scratch.element_size(), _stream(stream)),
            "combo_aggregation_divergence")
+    return rho_out
+
+
+def combo_aggregation_divergence_noalloc(models, mean_of, elem_bytes, weights, N, P, rho_out, stream=None):
+    """The same measurement for callers that cannot allocate device memory: the
+    partial sums go to a fixed 1 MiB array inside the library instead of a
+    caller-supplied scratch tensor.  At most 128 workers; all calls on a device
+    share that array, so issue them on one stream."""
+    _check(load().combo_aggregation_divergence_noalloc(_ptr(models), _ptr(mean_of), elem_bytes, _ptr(weights), N,
+                                                       P, _ptr(rho_out), _stream(stream)),
+           "combo_aggregation_divergence_noalloc")
     return rho_out
 
 

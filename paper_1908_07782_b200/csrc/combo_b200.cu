@@ -408,6 +408,31 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
     return COMBO_OK;
 }
 
+// ---------------------------------------------------------------- divergence without allocation
+// Fixed scratch for callers that cannot allocate device memory.  Every GPU that loads the
+// library holds this array (1 MiB) until the process exits.  In host code the array's name
+// is only a handle: the device address the kernels need comes from cudaGetSymbolAddress,
+// asked once per device with that device current.
+constexpr int kNoAllocMaxBlocks = 1024;
+static __device__ __align__(256) double g_noalloc_scratch[(size_t)kNoAllocMaxBlocks * COMBO_NOALLOC_MAX_WORKERS];
+double* g_noalloc_ptr[64];
+
+combo_status noalloc_scratch(double** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return COMBO_ERR_UNSUPPORTED;
+    if (!g_noalloc_ptr[dev]) {
+        double* ptr = nullptr;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(fixed scratch)");
+        if (!ptr) return COMBO_ERR_CUDA;
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return COMBO_OK;
+}
+
 // Streams and events of the host-memory entry point, created on its first call on a device.
 constexpr int kPipeChunks = 16;
 struct HostPipe {
@@ -609,6 +634,21 @@ combo_status combo_aggregation_divergence(const void* models, const void* mean_o
                            scratch_bytes, stream);
 }
 
+combo_status combo_aggregation_divergence_noalloc(const void* models, const void* mean_of, int elem_bytes,
+                                                  const float* weights, int N, int64_t P, double* rho_out,
+                                                  void* stream) {
+    if (N > COMBO_NOALLOC_MAX_WORKERS) {
+        snprintf(t_cuda_err, sizeof(t_cuda_err), "N = %d exceeds the fixed scratch (at most %d workers)", N,
+                 COMBO_NOALLOC_MAX_WORKERS);
+        return COMBO_ERR_TOO_LARGE;
+    }
+    double* scratch = nullptr;
+    combo_status rc = noalloc_scratch(&scratch);
+    if (rc != COMBO_OK) return rc;
+    return divergence_impl(models, mean_of, elem_bytes, weights, N, P, rho_out, scratch,
+                           sizeof(double) * (size_t)kNoAllocMaxBlocks * COMBO_NOALLOC_MAX_WORKERS, stream);
+}
+
 combo_status combo_device_status(void) {
     int v = 0;
     cudaError_t e = cudaDeviceSynchronize();
@@ -641,6 +681,7 @@ const char* combo_status_string(combo_status status) {
         case COMBO_ERR_UNSUPPORTED: return "device is not compute capability 10.x";
         case COMBO_ERR_CUDA: return "CUDA error";
         case COMBO_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        case COMBO_ERR_TOO_LARGE: return "size exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

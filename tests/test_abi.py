@@ -29,8 +29,8 @@ def test_library_builds_and_exports_every_declared_symbol():
 def test_status_strings_and_version():
     lib = combo.load()
     assert combo.combo_version() >= 100
-    seen = {lib.combo_status_string(i).decode() for i in range(6)}
-    assert len(seen) == 6 and "ok" in seen
+    seen = {lib.combo_status_string(i).decode() for i in range(7)}
+    assert len(seen) == 7 and "ok" in seen
     assert lib.combo_status_string(77).decode() == "unknown status"
 
 
