@@ -344,42 +344,61 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
     p.narr = two ? 2 : 1;
 
     int nblocks = 0;
-    // staged path: 16-byte aligned rows, at most 256 workers, two stages must fit
+    // staged path: rows at least 4-byte aligned, at most 256 workers, two stages must fit
     const long long pitch_bytes = P * EB;
-    const bool aligned = (pitch_bytes % 16) == 0 && aligned16(models) && aligned16(p.src);
-    if (t_force_path != 1 && aligned && N <= combo::kDivMaxStagedN && (long long)N * P >= (1 << 16) &&
-        (unsigned long long)P + 256 < (1ull << 31)) {
+    const int m = 16 / gcd_int(16, pitch_bytes % 16 == 0 ? 16 : pitch_bytes % 16);   // row classes
+    const bool word = m > 1;
+    if (t_force_path != 1 && (pitch_bytes % 4) == 0 && aligned16(models) && aligned16(p.src) &&
+        N <= combo::kDivMaxStagedN && (long long)N * P >= (1 << 16) && (unsigned long long)P + 256 < (1ull << 31) &&
+        (unsigned long long)m * (unsigned long long)pitch_bytes < (1ull << 40) && 2 * m <= 32) {
         const int V = 16 / EB;
-        const int G = combo::kConsumerThreads / (combo::kDivTile / V);
-        p.row_bytes = combo::kDivTile * EB;
         const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
         p.coef_off = header;
-        p.part_off = p.coef_off + round_up((unsigned)N * 4u, 128);
-        p.mean_off = p.part_off + (unsigned)G * combo::kDivTile * 4u;
+        p.rowoff_off = p.coef_off + round_up((unsigned)N * 4u, 128);
+        p.part_off = p.rowoff_off + round_up((unsigned)N * 4u, 128);
+        p.mean_off = p.part_off + (unsigned)combo::kConsumerThreads * V * 4u;   // G * PSTR floats at most
         p.stage_off = p.mean_off + combo::kDivTile * 4u;
-        p.stage_bytes = (unsigned)(p.narr * N * p.row_bytes);
+        p.m = m;
         const long long budget = (long long)dev->smem_optin - p.stage_off - 256;
-        const int fit = (int)(budget / p.stage_bytes);
-        int stages = (int)((112 * 1024) / p.stage_bytes);
-        if (stages < 2) stages = 2;
-        if (stages > combo::kMaxStages) stages = combo::kMaxStages;
-        if (stages > fit) stages = fit;
+        // tile and box: the widest of which two stages fit; with row phases one box of 256
+        int TC = 0, box = 0;
+        if (word) {
+            for (int c = combo::kDivTile; c >= 64; c >>= 1)
+                if (2LL * p.narr * N * c * EB <= budget) { TC = c - V; box = c; break; }
+        } else {
+            for (int c = combo::kDivTile; c >= 64; c >>= 1)
+                if (2LL * p.narr * N * c * EB <= budget) { TC = box = c; break; }
+        }
         combo::TileMaps maps;
-        if (stages >= 2 &&
-            encode_class_map(&maps.map[0][0], p.models, EB, 0, 1, N, P, P, combo::kDivTile) &&
-            (!two || encode_class_map(&maps.map[1][0], p.src, EB, 0, 1, N, P, P, combo::kDivTile))) {
+        bool ok = TC > 0;
+        for (int a = 0; ok && a < p.narr; ++a)
+            for (int j = 0; ok && j < m && j < N; ++j)
+                ok = encode_class_map(&maps.map[a][j], a == 0 ? p.models : p.src, EB, j, m, N, P, P, box);
+        if (ok) {
+            p.row_bytes = box * EB;
+            p.stage_bytes = (unsigned)(p.narr * N * p.row_bytes);
+            const int fit = (int)(budget / p.stage_bytes);
+            int stages = (int)((112 * 1024) / p.stage_bytes);
+            if (stages < 2) stages = 2;
+            if (stages > combo::kMaxStages) stages = combo::kMaxStages;
+            if (stages > fit) stages = fit;
             p.stages = stages;
-            p.n_tiles = (P + combo::kDivTile - 1) / combo::kDivTile;
+            p.n_tiles = (P + TC - 1) / TC;
             nblocks = (int)(p.n_tiles < dev->sms ? p.n_tiles : dev->sms);
-            const size_t smem = (size_t)p.stage_off + (size_t)stages * p.stage_bytes;
-            cudaError_t e;
-            if (EB == 4) {
-                e = cudaFuncSetAttribute(combo::k_divergence_staged<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                if (e == cudaSuccess) combo::k_divergence_staged<4><<<nblocks, combo::kStagedThreads, smem, st>>>(p, maps);
-            } else {
-                e = cudaFuncSetAttribute(combo::k_divergence_staged<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                if (e == cudaSuccess) combo::k_divergence_staged<2><<<nblocks, combo::kStagedThreads, smem, st>>>(p, maps);
-            }
+            const size_t smem = (size_t)p.stage_off + (size_t)stages * p.stage_bytes + 16;
+            cudaError_t e = cudaErrorInvalidValue;
+#define COMBO_DIV_LAUNCH(EBV, TCV, WV)                                                                          \
+    if (EB == EBV && TC == TCV && word == WV) {                                                                 \
+        e = cudaFuncSetAttribute(combo::k_divergence_staged<EBV, TCV, WV>,                                      \
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);                       \
+        if (e == cudaSuccess)                                                                                   \
+            combo::k_divergence_staged<EBV, TCV, WV><<<nblocks, combo::kStagedThreads, smem, st>>>(p, maps);    \
+    }
+            COMBO_DIV_LAUNCH(4, 256, false) COMBO_DIV_LAUNCH(4, 128, false) COMBO_DIV_LAUNCH(4, 64, false)
+            COMBO_DIV_LAUNCH(2, 256, false) COMBO_DIV_LAUNCH(2, 128, false) COMBO_DIV_LAUNCH(2, 64, false)
+            COMBO_DIV_LAUNCH(4, 252, true) COMBO_DIV_LAUNCH(4, 124, true) COMBO_DIV_LAUNCH(4, 60, true)
+            COMBO_DIV_LAUNCH(2, 248, true) COMBO_DIV_LAUNCH(2, 120, true) COMBO_DIV_LAUNCH(2, 56, true)
+#undef COMBO_DIV_LAUNCH
             if (e == cudaSuccess) e = cudaGetLastError();
             if (e != cudaSuccess) return cuda_fail(e, "divergence launch");
             t_last_path = 2;

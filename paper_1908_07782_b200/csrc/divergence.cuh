@@ -6,7 +6,7 @@
 //                        aggregation kernel; per tile: (A) column means from the staged
 //                        block, (B) warp-per-row sums of squared deviations, carried in
 //                        binary64 registers across the CTA's tiles
-//   k_divergence_direct  fallback for rows that are not 16-byte aligned or N > 256:
+//   k_divergence_direct  fallback for rows that are not even 4-byte aligned or N > 256:
 //                        thread per column, two passes through L1/L2
 //   k_divergence_finish  sums the per-CTA partial sums in block order and takes the root
 //
@@ -19,7 +19,7 @@ namespace combo {
 
 constexpr int kDivSlots = 16;                          // rows a consumer warp can own
 constexpr int kDivMaxStagedN = kDivSlots * kConsumerWarps;
-constexpr int kDivTile = 256;                          // columns per tile = one TMA box
+constexpr int kDivTile = 256;                          // widest tile in columns = one TMA box
 
 struct DivParams {
     const unsigned char* models;
@@ -27,23 +27,31 @@ struct DivParams {
     const float* weights;
     double* partial;               // scratch [grid][N]
     long long pitch, width, n_tiles;
-    int N, narr, stages, row_bytes;
-    unsigned coef_off, part_off, mean_off, stage_off, stage_bytes;
+    int N, narr, m, stages, row_bytes;
+    unsigned coef_off, rowoff_off, part_off, mean_off, stage_off, stage_bytes;
 };
 
-template <int EB>
+// TC = columns per tile.  Rows that are 16-byte aligned: 256, 128 or 64 (the widest of
+// which two stages fit), threads work on 128-bit vectors.  WORD: rows whose pitch is only a
+// multiple of 4 bytes are staged per row class with their phase (see the aggregation
+// kernel), TC = 256 - 16/e, and threads work on 4-byte words at the row's phase.
+template <int EB, int TC, bool WORD>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
-    constexpr int V = ElemOps<EB>::V;
-    constexpr int NV = kDivTile / V;                   // vectors per row per tile
-    constexpr int G = kConsumerThreads / NV;           // row groups of phase A
+    constexpr int UB = WORD ? 4 : 16;                  // bytes a thread takes at a time
+    constexpr int EPU = UB / EB;                       // elements in them
+    constexpr int NU = TC * EB / UB;                   // such units per row per tile
+    constexpr int NUP = NU <= 16 ? 16 : NU <= 32 ? 32 : NU <= 64 ? 64 : NU <= 128 ? 128 : 256;
+    constexpr int G = kConsumerThreads / NUP;          // row groups of phase A
+    constexpr int PSTR = NUP * EPU;                    // floats per row group in `part`
     extern __shared__ __align__(128) unsigned char smem[];
     StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = p.N, stages = p.stages;
     float* coef = reinterpret_cast<float*>(smem + p.coef_off);     // c_j = |D_j| / sum |D|
-    float* part = reinterpret_cast<float*>(smem + p.part_off);     // [G][kDivTile]
-    float* mean = reinterpret_cast<float*>(smem + p.mean_off);     // [kDivTile]
+    int* rowoff = reinterpret_cast<int*>(smem + p.rowoff_off);     // staged byte offset of worker j's tile part
+    float* part = reinterpret_cast<float*>(smem + p.part_off);     // [G][PSTR]
+    float* mean = reinterpret_cast<float*>(smem + p.mean_off);     // [TC]
     const int block_bytes = N * p.row_bytes;
 
     if (tid == 0) {
@@ -54,19 +62,30 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
         mbar_init(smem_u32(&hdr->csync), kConsumerWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // coefficients: the denominator is summed in worker order by every thread alike
+    // coefficients (the denominator is summed in worker order by every thread alike) and
+    // where each worker's row sits in a stage: classes one after another, phase included
     {
         float den = 0.0f;
         for (int j = 0; j < N; ++j) den = __fadd_rn(den, p.weights ? p.weights[j] : 1.0f);
-        for (int j = tid; j < N; j += kStagedThreads) coef[j] = __fdiv_rn(p.weights ? p.weights[j] : 1.0f, den);
+        for (int j = tid; j < N; j += kStagedThreads) {
+            coef[j] = __fdiv_rn(p.weights ? p.weights[j] : 1.0f, den);
+            const int jc = j % p.m;
+            int base = 0;
+            for (int q = 0; q < jc; ++q) base += (N - q + p.m - 1) / p.m;
+            rowoff[j] = (base + j / p.m) * p.row_bytes + (int)(((long long)j * p.pitch * EB) & 15);
+        }
     }
     __syncthreads();
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        const bool issuer = lane < p.narr;
-        const CUtensorMap* my_map = &maps.map[issuer ? lane : 0][0];
+        const int a = lane / p.m, j = lane - a * p.m;
+        const bool issuer = lane < p.narr * p.m && j < N;
+        int class_base = 0;
+        for (int q = 0; q < j; ++q) class_base += (N - q + p.m - 1) / p.m;
+        const CUtensorMap* my_map = &maps.map[issuer ? a : 0][issuer ? j : 0];
         if (issuer) asm volatile("prefetch.tensormap [%0];" ::"l"(my_map) : "memory");
+        const uint32_t my_dst_off = (uint32_t)(a * block_bytes + class_base * p.row_bytes);
         long long n = 0;
         for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % stages);
@@ -76,8 +95,8 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
             if (lane == 0) mbar_arrive_expect_tx(bar, p.stage_bytes);
             __syncwarp();
             if (issuer)
-                tma_load_2d(smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) + lane * block_bytes, my_map,
-                            (int)(tile * kDivTile), 0, bar);
+                tma_load_2d(smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) + my_dst_off, my_map,
+                            (int)(tile * TC), 0, bar);
         }
         if (lane == 0) {
             const long long first = n > stages ? n - stages : 0;
@@ -94,10 +113,23 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
     const int ctid = tid - 32;
     uint32_t csync_phase = 0;
     const uint32_t csync = smem_u32(&hdr->csync);
-    const int av = ctid % NV, ag = ctid / NV;           // phase A: vector and row group
+    const int au = ctid % NUP, ag = ctid / NUP;         // phase A: unit and row group
     double acc[kDivSlots];
 #pragma unroll
     for (int s = 0; s < kDivSlots; ++s) acc[s] = 0.0;
+
+    // one unit of a staged row as EPU binary32 values
+    auto load_unit = [](const unsigned char* q, float (&x)[EPU]) {
+        if constexpr (!WORD) {
+            GroupLoad<EB, 16>::run(q, x);
+        } else if constexpr (EB == 4) {
+            x[0] = *reinterpret_cast<const float*>(q);
+        } else {
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(q);
+            x[0] = bf16_widen(w & 0xffffu);
+            x[1] = __uint_as_float(w & 0xffff0000u);
+        }
+    };
 
     long long n = 0;
     for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
@@ -109,25 +141,25 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
 
         // (A) weighted column sums of this thread's row group; columns past the end of the
         // rows were zero-filled by the TMA unit and contribute nothing anywhere below
-        {
-            float a[V];
+        if (au < NU) {
+            float a[EPU];
 #pragma unroll
-            for (int i = 0; i < V; ++i) a[i] = 0.0f;
+            for (int i = 0; i < EPU; ++i) a[i] = 0.0f;
             for (int j = ag; j < N; j += G) {
-                float x[V];
-                GroupLoad<EB, 16>::run(xsrc + (size_t)j * p.row_bytes + av * 16, x);
+                float x[EPU];
+                load_unit(xsrc + rowoff[j] + au * UB, x);
                 const float c = coef[j];
 #pragma unroll
-                for (int i = 0; i < V; ++i) a[i] = fmaf(c, x[i], a[i]);
+                for (int i = 0; i < EPU; ++i) a[i] = fmaf(c, x[i], a[i]);
             }
 #pragma unroll
-            for (int i = 0; i < V; ++i) part[ag * kDivTile + av * V + i] = a[i];
+            for (int i = 0; i < EPU; ++i) part[ag * PSTR + au * EPU + i] = a[i];
         }
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(14); return; }
-        if (ctid < kDivTile) {
+        if (ctid < TC) {
             float m = 0.0f;
 #pragma unroll
-            for (int g = 0; g < G; ++g) m = __fadd_rn(m, part[g * kDivTile + ctid]);
+            for (int g = 0; g < G; ++g) m = __fadd_rn(m, part[g * PSTR + ctid]);
             mean[ctid] = m;
         }
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(15); return; }
@@ -138,14 +170,14 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
             const int i = cw + sl * kConsumerWarps;
             if (i < N) {
                 float ssum = 0.0f;
+                const unsigned char* row = stage + rowoff[i];
 #pragma unroll
-                for (int q = 0; q < NV / 32; ++q) {
-                    const int v = lane + 32 * q;
-                    float x[V];
-                    GroupLoad<EB, 16>::run(stage + (size_t)i * p.row_bytes + v * 16, x);
+                for (int u = lane; u < NU; u += 32) {
+                    float x[EPU];
+                    load_unit(row + u * UB, x);
 #pragma unroll
-                    for (int e = 0; e < V; ++e) {
-                        const float d = __fsub_rn(x[e], mean[v * V + e]);
+                    for (int e = 0; e < EPU; ++e) {
+                        const float d = __fsub_rn(x[e], mean[u * EPU + e]);
                         ssum = fmaf(d, d, ssum);
                     }
                 }

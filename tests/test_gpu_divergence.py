@@ -47,8 +47,11 @@ CASES = [
     (8, 100_000, torch.float32), (32, 65_536, torch.float32), (64, 40_004, torch.float32),
     (128, 30_008, torch.bfloat16), (16, 70_000, torch.bfloat16), (1, 5_000, torch.float32),
     (3, 1_000, torch.float32),                    # tiny: fallback kernel
-    (7, 100_001, torch.float32),                  # rows not 16-byte aligned: fallback kernel
-    (9, 100_001, torch.bfloat16),
+    (7, 100_001, torch.float32),                  # rows only 4-byte aligned: staged per row class
+    (40, 50_002, torch.bfloat16),                 # the same for bf16 (pitch = 4 mod 16 bytes)
+    (128, 20_010, torch.bfloat16),
+    (9, 100_001, torch.bfloat16),                 # odd bf16 pitch: fallback kernel
+    (64, 30_000, torch.float32),                  # two arrays of 64 rows: half-width tiles
     (200, 20_000, torch.float32),                 # too many rows for two staged tiles: fallback
     (300, 4_096, torch.bfloat16),                 # more than 256 workers
 ]
