@@ -1,0 +1,39 @@
+"""Randomised shapes: both aggregation kernels against the oracle and each other."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1908_07782_b200 as combo
+
+from gpu_util import DEV, check_against_oracle, gpu_aggregate
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes(seed):
+    rng = np.random.default_rng(1000 + seed)
+    dtype = torch.float32 if rng.random() < 0.6 else torch.bfloat16
+    N = int(rng.choice([2, 3, 5, 8, 13, 16, 31, 32, 48, 64, 96, 128, 160]))
+    R = int(rng.integers(0, min(N - 1, 9) + 1))
+    S = int(rng.choice([1, 2, 3, 4, 7, 8, 10, 16, 32]))
+    P = int(rng.integers(20_000, 400_000 // max(N // 16, 1)))
+    P += int(rng.integers(0, 16))                       # every alignment residue
+    fused = dtype == torch.float32 and rng.random() < 0.4
+    weighted = rng.random() < 0.5
+    g = torch.Generator().manual_seed(seed)
+    x = (torch.randn(N, P, generator=g) * 0.05).to(dtype).to(DEV)
+    grads = (torch.randn(N, P, generator=g) * 1e-3).to(DEV) if fused else None
+    w = torch.randint(500, 1501, (N,), generator=g).float().to(DEV) if weighted else None
+    idx_np = oracle.select_peers(seed, seed % 5, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV) if R > 0 else None
+    a, _ = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_STAGED)
+    b, _ = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_DIRECT)
+    assert torch.equal(a, b), (N, P, S, R, dtype, fused)
+    lo, hi = 0, min(P, 3000)
+    mid = P // 2
+    for (c0, c1) in ((lo, hi), (max(mid - 1500, 0), min(mid + 1500, P)), (max(P - 3000, 0), P)):
+        check_against_oracle(x[:, c0:c1].contiguous(), a[:, c0:c1].contiguous(), idx_np, S, R, weights=w,
+                             grads=grads[:, c0:c1].contiguous() if fused else None, lr=0.01, P=P, p_begin=c0)
+    combo.combo_device_status()
