@@ -90,7 +90,7 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
         for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % stages);
             const uint32_t ph = (uint32_t)((n / stages) & 1);
-            if (!mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(11); break; }
+            if (!mbar_wait_patient(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(11); break; }
             const uint32_t bar = smem_u32(&hdr->full[s]);
             if (lane == 0) mbar_arrive_expect_tx(bar, p.stage_bytes);
             __syncwarp();

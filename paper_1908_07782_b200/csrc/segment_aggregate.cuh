@@ -375,6 +375,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return false;
 }
+// The producer warp is always ahead of the consumers, so it spends the kernel waiting for a
+// free stage.  Spinning there would compete for issue slots with the consumer warps of the
+// same scheduler; it sleeps between polls instead (a stage is re-armed a tile ahead of its
+// use, so a fraction of a microsecond of wake-up latency costs nothing).
+__device__ __forceinline__ bool mbar_wait_patient(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+#pragma unroll 1
+    for (uint32_t it = 0; it < kWaitCap; ++it) {
+        asm volatile(
+            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        __nanosleep(256);
+    }
+    return false;
+}
 // Tiled 2-D TMA load of one box (x = element column, y = row of the class) into this CTA's
 // shared memory; completion bytes are counted on `bar`.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
@@ -505,7 +523,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % stages);
             const uint32_t ph = (uint32_t)((n / stages) & 1);
-            if (!mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); break; }
+            if (!mbar_wait_patient(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); break; }
             const long long t0 = tile * (long long)p.T;
             const uint32_t bar = smem_u32(&hdr->full[s]);
             if (lane == 0) {
@@ -631,23 +649,26 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
 
         int row = row_begin, xb = xb_begin;
         if (interior) {
-            // every unit is whole and lies in segment l0: the lean loop
+            // every unit is whole and lies in segment l0: the lean loop, rows outside, boxes inside
             RowCtx<RMAX> c;
-            int cur_row = -1;
-            unsigned char* orow = nullptr;
-            for (int u = u_begin; u < u_end; ++u) {
-                if (row != cur_row) {
-                    cur_row = row;
-                    load_entry<RMAX>(tab + (size_t)row * ENT, c);
-                    orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
-                }
-                const uint32_t ubase = stage_s + xb * block_bytes + lane * GB;
-                unsigned char* uout = orow + xb * box_payload;
+            const int nbx = p.nbx;
+            const unsigned char* ent = tab + (size_t)row * ENT;
+            unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
+            const uint32_t lane_base = stage_s + lane * GB;
+            int u = u_begin;
+            while (u < u_end) {
+                load_entry<RMAX>(ent, c);
+                for (; xb < nbx && u < u_end; ++xb, ++u) {
+                    const uint32_t ubase = lane_base + xb * block_bytes;
+                    unsigned char* uout = orow + xb * box_payload;
 #pragma unroll
-                for (int ch = 0; ch < CPB; ++ch)
-                    if (GB == 16 || ch * 512 < box_payload)
-                        item_fast<EB, GB, RMAX, (RT >= 0)>(ubase + ch * 512, c, R, uout + ch * 512, pmask[ch]);
-                if (++xb == p.nbx) { xb = 0; ++row; }
+                    for (int ch = 0; ch < CPB; ++ch)
+                        if (GB == 16 || ch * 512 < box_payload)
+                            item_fast<EB, GB, RMAX, (RT >= 0)>(ubase + ch * 512, c, R, uout + ch * 512, pmask[ch]);
+                }
+                xb = 0;
+                ent += ENT;
+                orow += pitch_bytes;
             }
         } else {
             // last tile of the rows, or a tile holding a segment boundary: element by element,
