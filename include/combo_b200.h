@@ -45,7 +45,7 @@ enum {
     COMBO_ERR_TOO_LARGE = 6       /* beyond the fixed limit of a no-allocation entry point */
 };
 
-/* Limits of this build. */
+/* Limits of this library version. */
 #define COMBO_MAX_WORKERS 8192    /* N */
 #define COMBO_MAX_SEGMENTS 65536  /* S */
 #define COMBO_NOALLOC_MAX_WORKERS 128   /* N of combo_aggregation_divergence_noalloc */
