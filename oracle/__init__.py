@@ -70,6 +70,14 @@ def _load():
     lib.oracle_divergence.restype = ctypes.c_int
     lib.oracle_divergence.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
                                       ctypes.c_int, ctypes.c_int64, ctypes.c_void_p]
+    lib.oracle_select_peers_active.restype = ctypes.c_int
+    lib.oracle_select_peers_active.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int, ctypes.c_int,
+                                               ctypes.c_int, ctypes.c_void_p, i32p]
+    lib.oracle_segment_aggregate_members.restype = ctypes.c_int
+    lib.oracle_segment_aggregate_members.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+                                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                                     ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                                     ctypes.c_void_p]
     _lib = lib
     return lib
 
@@ -201,3 +209,46 @@ def divergence(models, weights=None, mean_of=None) -> np.ndarray:
     if rc != 0:
         raise ValueError("oracle_divergence: invalid arguments")
     return rho
+
+
+def select_peers_active(seed, rnd, N, S, R, active=None) -> np.ndarray:
+    """Section 4.2: peers drawn from the ONLINE others only; rows of offline workers are -1."""
+    lib = _load()
+    idx = np.zeros((N, S, max(R, 0)), dtype=np.int32)
+    aptr = None
+    if active is not None:
+        active = np.ascontiguousarray(active, dtype=np.uint8)
+        aptr = active.ctypes.data
+    rc = lib.oracle_select_peers_active(seed, rnd, N, S, R, aptr,
+                                        idx.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)))
+    if rc != 0:
+        raise ValueError("oracle_select_peers_active: invalid arguments")
+    return idx
+
+
+def segment_aggregate_members(x, idx, S, R, weights=None, newcomer=None, ordered=False) -> np.ndarray:
+    """Eq. 3 with Section 4.2's provider sets: self unless a newcomer, plus the
+    non-negative idx entries.  binary64 result, or the fixed-order binary32 form."""
+    lib = _load()
+    elem = 4 if x.dtype == np.float32 else 2
+    xptr, P = _slab(x, elem)
+    N = x.shape[0]
+    wptr = None
+    if weights is not None:
+        weights = np.ascontiguousarray(weights, dtype=np.float32)
+        wptr = weights.ctypes.data
+    nptr = None
+    if newcomer is not None:
+        newcomer = np.ascontiguousarray(newcomer, dtype=np.uint8)
+        nptr = newcomer.ctypes.data
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    iptr = idx.ctypes.data if R > 0 else None
+    if ordered:
+        out = np.empty((N, P), dtype=np.float32 if elem == 4 else np.uint16)
+    else:
+        out = np.empty((N, P), dtype=np.float64)
+    rc = lib.oracle_segment_aggregate_members(xptr, elem, wptr, iptr, nptr, N, P, S, R, 1 if ordered else 0,
+                                              out.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle_segment_aggregate_members: invalid arguments")
+    return out

@@ -21,6 +21,12 @@
  *                                when S*R <= n-1), uniformity of the shuffle.
  *                                Its exact tables are PARITY UNPINNED by the
  *                                paper, which names no generator.
+ *   oracle_select_peers_active   equals oracle_select_peers when all are online;
+ *                                never an offline peer; same invariants on the
+ *                                online pool; offline rows are -1
+ *   oracle_segment_aggregate_members  equals oracle_segment_aggregate without
+ *                                newcomers / absent peers; exact rationals with
+ *                                them; a newcomer's own values never matter
  *   oracle_divergence            exact rational brute force of Eq. 7 on tiny
  *                                inputs, two-worker closed form, identical
  *                                models (zero), R = n-1 (zero, as the paper
@@ -297,5 +303,137 @@ int oracle_divergence(const void *models, const void *mean_of, int elem, const f
         }
     }
     for (int i = 0; i < N; ++i) rho[i] = sqrt(rho[i]);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* Dynamic workers (Section 4.2).                                      */
+/* (1) A worker that is offline is not pulled from: requests go to     */
+/*     "another worker", so the pool of a worker is the ONLINE others. */
+/*     Offline workers issue no requests: their rows are filled -1.    */
+/*     With every worker online this is oracle_select_peers exactly.   */
+/*     active: N bytes, non-zero = online; NULL = all online.          */
+/*     Requires R <= (number of online workers) - 1.                   */
+/* ------------------------------------------------------------------ */
+int oracle_select_peers_active(uint64_t seed, uint32_t round, int N, int S, int R,
+                               const uint8_t *active, int32_t *idx) {
+    if (N < 1 || S < 1 || R < 0) return 1;
+    int n_on = 0;
+    for (int v = 0; v < N; ++v) n_on += (!active || active[v]) ? 1 : 0;
+    if (R > 0 && R > n_on - 1) return 1;
+    if (R == 0) return 0;
+    int32_t *pool = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+    int32_t *perm = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+    int32_t *tmp = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+    int32_t *chosen = (int32_t *)malloc(sizeof(int32_t) * (size_t)R);
+    for (int w = 0; w < N; ++w) {
+        int32_t *rows = idx + (size_t)w * S * R;
+        if (active && !active[w]) {
+            for (int i = 0; i < S * R; ++i) rows[i] = -1;
+            continue;
+        }
+        int M = 0;
+        for (int v = 0; v < N; ++v)
+            if (v != w && (!active || active[v])) pool[M++] = v;
+        int pos = M;
+        uint32_t epoch = 0;
+        int opened = 0;
+        for (int l = 0; l < S; ++l) {
+            int nc = 0;
+            for (int r = 0; r < R; ++r) {
+                if (pos == M) {
+                    if (opened) ++epoch;
+                    opened = 1;
+                    memcpy(perm, pool, sizeof(int32_t) * (size_t)M);
+                    for (int t = M - 1; t >= 1; --t) {
+                        uint32_t u = oracle_rand32(seed, round, (uint32_t)w, epoch, (uint32_t)t);
+                        int j = (int)(((uint64_t)u * (uint64_t)(t + 1)) >> 32);
+                        int32_t s = perm[t]; perm[t] = perm[j]; perm[j] = s;
+                    }
+                    if (nc > 0) {
+                        int a = 0;
+                        for (int pass = 0; pass < 2; ++pass)
+                            for (int i = 0; i < M; ++i) {
+                                int taken = 0;
+                                for (int c = 0; c < nc; ++c) taken |= (chosen[c] == perm[i]);
+                                if (taken == pass) tmp[a++] = perm[i];
+                            }
+                        memcpy(perm, tmp, sizeof(int32_t) * (size_t)M);
+                    }
+                    pos = 0;
+                }
+                chosen[nc++] = perm[pos++];
+            }
+            qsort(chosen, (size_t)R, sizeof(int32_t), cmp_i32);
+            memcpy(rows + (size_t)l * R, chosen, sizeof(int32_t) * (size_t)R);
+        }
+    }
+    free(pool); free(perm); free(tmp); free(chosen);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* (2) Eq. 3 with the provider sets Section 4.2 allows:                */
+/*     P_l(w) = ({w} unless w is a newcomer) U {idx[w][l][r] >= 0}.    */
+/*     A new worker "pulls the segments and aggregates them as normal  */
+/*     only without its local model"; a negative idx entry is a pull   */
+/*     that found no online peer.  An empty P_l leaves the worker's    */
+/*     own values (reading: nothing to aggregate).                     */
+/*     newcomer: N bytes or NULL.  mode 0: binary64, quotient of sums, */
+/*     out = double; mode 1: the fixed-order binary32 form, out =      */
+/*     float (elem 4) or bf16 bits (elem 2).                           */
+/* ------------------------------------------------------------------ */
+int oracle_segment_aggregate_members(const void *in, int elem, const float *weights, const int32_t *idx,
+                                     const uint8_t *newcomer, int N, int64_t P, int S, int R, int mode,
+                                     void *out) {
+    if (N < 1 || P < 1 || S < 1 || R < 0 || (elem != 4 && elem != 2)) return 1;
+    int64_t L = oracle_segment_length(P, S);
+    int *prov = (int *)malloc(sizeof(int) * (size_t)(R + 1));
+    float *coef = (float *)malloc(sizeof(float) * (size_t)(R + 1));
+    for (int w = 0; w < N; ++w) {
+        for (int l = 0; l < S; ++l) {
+            int64_t a = (int64_t)l * L, b = a + L;
+            if (b > P) b = P;
+            if (a >= b) continue;
+            int np = 0;
+            if (!newcomer || !newcomer[w]) prov[np++] = w;
+            for (int r = 0; r < R; ++r) {
+                int k = idx[((size_t)w * S + l) * R + r];
+                if (k >= 0) prov[np++] = k;
+            }
+            if (np == 0) prov[np++] = w;
+            if (mode == 1) {
+                volatile float den = 0.0f;
+                for (int q = 0; q < np; ++q) {
+                    float D = weights ? weights[prov[q]] : 1.0f;
+                    den = (q == 0) ? D : den + D;
+                }
+                for (int q = 0; q < np; ++q) coef[q] = (weights ? weights[prov[q]] : 1.0f) / den;
+            }
+            for (int64_t p = a; p < b; ++p) {
+                size_t o = (size_t)w * (size_t)P + (size_t)p;
+                if (mode == 0) {
+                    double num = 0.0, den = 0.0;
+                    for (int q = 0; q < np; ++q) {
+                        double D = weights ? (double)weights[prov[q]] : 1.0;
+                        num += D * load_x(in, elem, (size_t)prov[q] * (size_t)P + (size_t)p);
+                        den += D;
+                    }
+                    ((double *)out)[o] = num / den;
+                } else {
+                    float acc = 0.0f;
+                    for (int q = 0; q < np; ++q) {
+                        size_t off = (size_t)prov[q] * (size_t)P + (size_t)p;
+                        float x = (elem == 4) ? ((const float *)in)[off] : bf16_to_f32(((const uint16_t *)in)[off]);
+                        if (q == 0) { volatile float prod = coef[0] * x; acc = prod; }
+                        else acc = fmaf(coef[q], x, acc);
+                    }
+                    if (elem == 4) ((float *)out)[o] = acc;
+                    else ((uint16_t *)out)[o] = oracle_f32_to_bf16_rne(acc);
+                }
+            }
+        }
+    }
+    free(prov); free(coef);
     return 0;
 }
