@@ -140,6 +140,35 @@ combo_status combo_segment_aggregate_cols(const void* params_in, const void* gra
                                           void* stream);
 
 /*
+ * Dynamic workers -- Section 4.2.
+ *
+ * combo_select_peers_online: a worker that is offline is not pulled from (the
+ * requester "resends the request to another worker"), so every online worker
+ * draws its peers from the ONLINE others only, by the same procedure as
+ * combo_select_peers (identical tables when all are online).  An offline worker
+ * issues no requests: its rows are filled with -1.  h_online: HOST array of N
+ * bytes, non-zero = online (membership is decided on the host); NULL = all
+ * online.  Requires R <= (online workers) - 1.
+ *
+ * combo_segment_aggregate_members: Eq. 3 with the provider set
+ *   P_l(w) = ({w} unless w is a newcomer) U { idx[w][l][r] : idx[w][l][r] >= 0 }.
+ * A new worker "pulls the segments and aggregates them as normal only without
+ * its local model", so its own row is never read; a negative idx entry is a
+ * pull that found no online peer.  A worker left with no provider (an offline
+ * worker's -1 rows) keeps its own values.  h_newcomer: HOST array of N bytes,
+ * non-zero = newcomer, or NULL.  Same arithmetic and order as
+ * combo_segment_aggregate (providers in the order self, peers ascending); all
+ * entry points above accept negative idx entries in the same way.  Rows that are
+ * read must hold finite values.
+ */
+combo_status combo_select_peers_online(uint64_t seed, uint32_t round, int N, int S, int R,
+                                       const uint8_t* h_online, int32_t* idx_out, void* stream);
+combo_status combo_segment_aggregate_members(const void* params_in, void* params_out, int elem_bytes,
+                                             const float* weights, const int32_t* idx,
+                                             const uint8_t* h_newcomer, int N, int64_t P, int S, int R,
+                                             void* stream);
+
+/*
  * Checks an idx table on the device: every entry in [0,N), != its worker,
  * each (w,l) row strictly ascending.  dev_flag: device int32, set to 0 first,
  * then to 1 + (index of an offending entry) if any check fails.

@@ -47,6 +47,8 @@ def load():
         "combo_segment_aggregate_cols": [vp, vp, f32, vp, i32, vp, vp, i32, i64, i32, i32, i64, i64,
                                          i64, vp],
         "combo_validate_idx": [vp, i32, i32, i32, vp, vp],
+        "combo_select_peers_online": [u64, u32, i32, i32, i32, vp, vp, vp],
+        "combo_segment_aggregate_members": [vp, vp, i32, vp, vp, vp, i32, i64, i32, i32, vp],
         "combo_round_host": [vp, vp, f32, vp, i32, vp, u64, u32, i32, i32, i64, i32, i32, vp, vp, vp,
                              vp, vp, vp, vp],
         "combo_aggregation_divergence": [vp, vp, i32, vp, i32, i64, vp, vp, ctypes.c_size_t, vp],
@@ -129,6 +131,33 @@ def combo_segment_aggregate_cols(params_in, grads, lr, params_out, elem_bytes, w
                                                elem_bytes, _ptr(weights), _ptr(idx), N, P_total, S, R,
                                                p_begin, width, pitch, _stream(stream)),
            "combo_segment_aggregate_cols")
+    return params_out
+
+
+def _host_bytes(flags, N):
+    """N flag bytes in host memory for the C side (None stays NULL)."""
+    if flags is None:
+        return None, None
+    buf = (ctypes.c_uint8 * N)(*[1 if bool(f) else 0 for f in flags])
+    return buf, ctypes.cast(buf, ctypes.c_void_p)
+
+
+def combo_select_peers_online(seed, rnd, N, S, R, online, idx_out, stream=None):
+    """Section 4.2: peers drawn from the online others only; ``online`` is a host
+    sequence of N flags (None = all online).  Offline workers' rows become -1."""
+    keep, ptr = _host_bytes(online, N)
+    _check(load().combo_select_peers_online(seed, rnd, N, S, R, ptr, _ptr(idx_out), _stream(stream)),
+           "combo_select_peers_online")
+    return idx_out
+
+
+def combo_segment_aggregate_members(params_in, params_out, weights, idx, newcomer, N, P, S, R, stream=None):
+    """Eq. 3 where newcomers (host sequence of N flags, or None) aggregate without their
+    own model and negative idx entries are skipped."""
+    keep, ptr = _host_bytes(newcomer, N)
+    _check(load().combo_segment_aggregate_members(_ptr(params_in), _ptr(params_out), params_in.element_size(),
+                                                  _ptr(weights), _ptr(idx), ptr, N, P, S, R, _stream(stream)),
+           "combo_segment_aggregate_members")
     return params_out
 
 

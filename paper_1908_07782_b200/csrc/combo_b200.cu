@@ -261,7 +261,8 @@ cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo
 
 combo_status aggregate_cols(const void* in, const void* grads, float lr, void* out, int EB,
                             const float* weights, const int32_t* idx, int N, long long P_total, int S, int R,
-                            long long p_begin, long long width, long long pitch, void* stream) {
+                            long long p_begin, long long width, long long pitch, void* stream,
+                            const uint8_t* h_newcomer = nullptr) {
     if (EB != 4 && EB != 2) return COMBO_ERR_INVALID_ARG;
     if (N < 1 || N > COMBO_MAX_WORKERS || S < 1 || S > COMBO_MAX_SEGMENTS || R < 0 || R > N - 1)
         return COMBO_ERR_INVALID_ARG;
@@ -291,6 +292,9 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
     p.L = (P_total + S - 1) / S;
     p.N = N; p.S = S; p.R = R;
     p.lr = lr;
+    if (h_newcomer)
+        for (int v = 0; v < N; ++v)
+            if (h_newcomer[v]) p.newcomer.w[v >> 5] |= 1u << (v & 31);
     const bool sgd = grads != nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
@@ -484,22 +488,36 @@ combo_status host_pipe(HostPipe** out) {
 }
 
 combo_status select_peers_impl(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* idx_out,
-                               cudaStream_t st) {
+                               cudaStream_t st, const uint8_t* h_online = nullptr) {
     if (N < 1 || N > COMBO_MAX_WORKERS || S < 1 || S > COMBO_MAX_SEGMENTS || R < 0 || R > N - 1)
         return COMBO_ERR_INVALID_ARG;
+    combo::WorkerBits bits;
+    memset(&bits, 0, sizeof(bits));
+    if (h_online) {
+        int n_on = 0;
+        for (int v = 0; v < N; ++v)
+            if (h_online[v]) { bits.w[v >> 5] |= 1u << (v & 31); ++n_on; }
+        if (R > 0 && R > n_on - 1) return COMBO_ERR_INVALID_ARG;
+    }
     if (R == 0) return COMBO_OK;
     if (!idx_out) return COMBO_ERR_INVALID_ARG;
     DeviceInfo* dev = nullptr;
     combo_status rc = device_info(&dev);
     if (rc != COMBO_OK) return rc;
     const size_t smem = combo::select_peers_smem_bytes(N);
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(combo::k_select_peers, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(select_peers)");
+    cudaError_t e = cudaSuccess;
+    if (h_online) {
+        if (smem > 48 * 1024)
+            e = cudaFuncSetAttribute(combo::k_select_peers<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess)
+            combo::k_select_peers<true><<<N, combo::kSelectThreads, smem, st>>>(seed, round, N, S, R, idx_out, bits);
+    } else {
+        if (smem > 48 * 1024)
+            e = cudaFuncSetAttribute(combo::k_select_peers<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess)
+            combo::k_select_peers<false><<<N, combo::kSelectThreads, smem, st>>>(seed, round, N, S, R, idx_out, bits);
     }
-    combo::k_select_peers<<<N, combo::kSelectThreads, smem, st>>>(seed, round, N, S, R, idx_out);
-    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "select_peers launch");
     return COMBO_OK;
 }
@@ -540,6 +558,18 @@ combo_status combo_segment_aggregate_cols(const void* params_in, const void* gra
                                           int64_t pitch, void* stream) {
     return aggregate_cols(params_in, grads, lr, params_out, elem_bytes, weights, idx, N, P_total, S, R, p_begin,
                           width, pitch, stream);
+}
+
+combo_status combo_select_peers_online(uint64_t seed, uint32_t round, int N, int S, int R, const uint8_t* h_online,
+                                       int32_t* idx_out, void* stream) {
+    return select_peers_impl(seed, round, N, S, R, idx_out, static_cast<cudaStream_t>(stream), h_online);
+}
+
+combo_status combo_segment_aggregate_members(const void* params_in, void* params_out, int elem_bytes,
+                                             const float* weights, const int32_t* idx, const uint8_t* h_newcomer,
+                                             int N, int64_t P, int S, int R, void* stream) {
+    return aggregate_cols(params_in, nullptr, 0.0f, params_out, elem_bytes, weights, idx, N, P, S, R, 0, P, P, stream,
+                          h_newcomer);
 }
 
 combo_status combo_validate_idx(const int32_t* idx, int N, int S, int R, void* stream, int32_t* dev_flag) {

@@ -49,6 +49,13 @@ constexpr int kMaxBoxes = 8;              // x-boxes per tile
 constexpr uint32_t kWaitCap = 1u << 23;   // polls before a wait is declared dead
 constexpr uint32_t kWaitHintNs = 1000;    // time a single poll may stay suspended
 
+// One flag per worker (up to COMBO_MAX_WORKERS), passed by value (Section 4.2: online /
+// offline workers, newcomers).
+struct WorkerBits {
+    uint32_t w[256];
+    __host__ __device__ bool get(int i) const { return (w[i >> 5] >> (i & 31)) & 1u; }
+};
+
 struct AggParams {
     const unsigned char* in;
     const unsigned char* grads;
@@ -71,6 +78,7 @@ struct AggParams {
     unsigned tab_off;    // byte offset of the coefficient table in shared memory
     unsigned stage_off;  // byte offset of stage 0
     unsigned stage_bytes;
+    WorkerBits newcomer; // workers that aggregate without their own model (Section 4.2)
 };
 
 // Tensor maps of one launch: [array][class], array 0 = parameters, 1 = gradients.
@@ -268,6 +276,38 @@ __device__ __forceinline__ float direct_x(const AggParams& p, int k, long long c
     return x;
 }
 
+// Providers of (worker w, segment l) in the fixed order: the worker itself unless it is a
+// newcomer, then its peers ascending (negative entries are absent); the worker alone if that
+// leaves nobody.  Returns the count; prov needs room for R+1 entries only when R is small,
+// so callers iterate with this helper instead of storing the list.
+struct ProviderIter {
+    const int32_t* peers;
+    int w, R, pos;      // pos: -1 = self pending, 0..R-1 = next peer slot
+    bool self_in;
+    __device__ ProviderIter(const AggParams& p, int w_, long long l)
+        : peers(p.R > 0 ? p.idx + ((size_t)w_ * p.S + (size_t)l) * (size_t)p.R : nullptr), w(w_), R(p.R), pos(-1) {
+        self_in = !p.newcomer.get(w_);
+        if (!self_in) {
+            bool any = false;
+            for (int r = 0; r < R; ++r) any |= peers[r] >= 0;
+            if (!any) self_in = true;
+        }
+    }
+    __device__ void rewind() { pos = -1; }
+    // next provider or -1
+    __device__ int next() {
+        if (pos < 0) {
+            pos = 0;
+            if (self_in) return w;
+        }
+        while (pos < R) {
+            const int k = peers[pos++];
+            if (k >= 0) return k;
+        }
+        return -1;
+    }
+};
+
 template <int EB, bool SGD>
 __global__ void __launch_bounds__(256) k_direct(const AggParams p) {
     constexpr int V = ElemOps<EB>::V;
@@ -284,26 +324,18 @@ __global__ void __launch_bounds__(256) k_direct(const AggParams p) {
         if (lo >= hi) continue;
         const long long l_lo = (p.p_begin + lo) / p.L, l_hi = (p.p_begin + hi - 1) / p.L;
         if (hi - lo == V && l_lo == l_hi && rows_aligned) {
-            const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l_lo) * (size_t)p.R;
-            const float dw = p.weights ? p.weights[w] : 1.0f;
-            float den = dw;
-            for (int r = 0; r < p.R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
-            float acc[V], x[V];
-            {
-                const size_t off = ((size_t)w * (size_t)p.pitch + (size_t)c0) * EB;
-                GroupLoad<EB, 16>::run(p.in + off, x);
-                if (SGD) {
-                    float gx[V];
-                    GroupLoad<EB, 16>::run(p.grads + off, gx);
-#pragma unroll
-                    for (int i = 0; i < V; ++i) x[i] = fmaf(-p.lr, gx[i], x[i]);
-                }
-                const float c = __fdiv_rn(dw, den);
-#pragma unroll
-                for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(c, x[i]);
+            ProviderIter pi(p, w, l_lo);
+            float den = 0.0f;
+            bool first = true;
+            for (int k = pi.next(); k >= 0; k = pi.next()) {
+                const float D = p.weights ? p.weights[k] : 1.0f;
+                den = first ? D : __fadd_rn(den, D);
+                first = false;
             }
-            for (int r = 0; r < p.R; ++r) {
-                const int k = peers[r];
+            pi.rewind();
+            float acc[V], x[V];
+            first = true;
+            for (int k = pi.next(); k >= 0; k = pi.next()) {
                 const size_t off = ((size_t)k * (size_t)p.pitch + (size_t)c0) * EB;
                 GroupLoad<EB, 16>::run(p.in + off, x);
                 if (SGD) {
@@ -313,21 +345,34 @@ __global__ void __launch_bounds__(256) k_direct(const AggParams p) {
                     for (int i = 0; i < V; ++i) x[i] = fmaf(-p.lr, gx[i], x[i]);
                 }
                 const float c = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                if (first) {
 #pragma unroll
-                for (int i = 0; i < V; ++i) acc[i] = fmaf(c, x[i], acc[i]);
+                    for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(c, x[i]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < V; ++i) acc[i] = fmaf(c, x[i], acc[i]);
+                }
+                first = false;
             }
             ElemOps<EB>::store_vec(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c0) * EB, acc);
         } else {
             for (long long c = lo; c < hi; ++c) {
-                const long long l = (p.p_begin + c) / p.L;
-                const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)p.R;
-                const float dw = p.weights ? p.weights[w] : 1.0f;
-                float den = dw;
-                for (int r = 0; r < p.R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
-                float acc = __fmul_rn(__fdiv_rn(dw, den), direct_x<EB, SGD>(p, w, c));
-                for (int r = 0; r < p.R; ++r) {
-                    const int k = peers[r];
-                    acc = fmaf(__fdiv_rn(p.weights ? p.weights[k] : 1.0f, den), direct_x<EB, SGD>(p, k, c), acc);
+                ProviderIter pi(p, w, (p.p_begin + c) / p.L);
+                float den = 0.0f;
+                bool first = true;
+                for (int k = pi.next(); k >= 0; k = pi.next()) {
+                    const float D = p.weights ? p.weights[k] : 1.0f;
+                    den = first ? D : __fadd_rn(den, D);
+                    first = false;
+                }
+                pi.rewind();
+                float acc = 0.0f;
+                first = true;
+                for (int k = pi.next(); k >= 0; k = pi.next()) {
+                    const float cf = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                    const float x = direct_x<EB, SGD>(p, k, c);
+                    acc = first ? __fmul_rn(cf, x) : fmaf(cf, x, acc);
+                    first = false;
                 }
                 ElemOps<EB>::store(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c) * EB, acc);
             }
@@ -584,11 +629,20 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
             float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
             int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
-            const float dw = p.weights ? p.weights[w] : 1.0f;
-            float den = dw;
-            for (int r = 0; r < R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
-            for (int r = 0; r <= R; ++r) {
-                const int k = (r == 0) ? w : peers[r - 1];
+            // providers in the fixed order: the worker itself (unless it is a newcomer), then
+            // the peers ascending; a negative entry is a pull that found no online peer
+            int prov[RMAX + 1];
+            int np = 0;
+            if (!p.newcomer.get(w)) prov[np++] = w;
+            for (int r = 0; r < R; ++r) {
+                const int k = peers[r];
+                if (k >= 0) prov[np++] = k;
+            }
+            if (np == 0) prov[np++] = w;                 // nothing to aggregate: keep the own values
+            float den = p.weights ? p.weights[prov[0]] : 1.0f;
+            for (int t = 1; t < np; ++t) den = __fadd_rn(den, p.weights ? p.weights[prov[t]] : 1.0f);
+            for (int r = 0; r < np; ++r) {
+                const int k = prov[r];
                 cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
                 // staged row of worker k: classes are stored one after another
                 const int jk = k % p.m;
@@ -597,7 +651,8 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                 const int phase = (int)(((long long)k * p.pitch * EB) & 15);
                 po[r] = (base + k / p.m) * p.row_bytes + phase;
             }
-            for (int r = R + 1; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
+            // unused slots: coefficient zero on a row that is known to hold finite values
+            for (int r = np; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
         }
     }
     };

@@ -10,6 +10,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "segment_aggregate.cuh"
+
 namespace combo {
 
 // splitmix64 output function (Steele, Lea, Flood 2014) and its increment.
@@ -25,19 +27,45 @@ __device__ __forceinline__ uint64_t splitmix_step(uint64_t state) {
 constexpr int kSelectThreads = 128;
 
 __host__ __device__ inline size_t select_peers_smem_bytes(int N) {
-    // perm[N-1] + aux[N-1] as int32, mark[N] as bytes, rounded up
-    return (size_t)(N > 1 ? N - 1 : 1) * 8 + (size_t)N + 16;
+    // perm[N] + aux[N] + pool[N] as int32, mark[N] as bytes, rounded up
+    return (size_t)N * 12 + (size_t)N + 16;
 }
 
+// MASKED: the pool of worker w is the ONLINE others (ascending); an offline worker issues
+// no requests and its rows are filled with -1.
+template <bool MASKED>
 __global__ void __launch_bounds__(kSelectThreads)
-k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __restrict__ idx) {
+k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __restrict__ idx,
+               const WorkerBits online) {
     extern __shared__ __align__(16) unsigned char sp_smem[];
     const int w = blockIdx.x;
-    const int M = N - 1;
     int32_t* perm = reinterpret_cast<int32_t*>(sp_smem);
-    int32_t* aux = perm + M;
-    uint8_t* mark = reinterpret_cast<uint8_t*>(aux + M);
+    int32_t* aux = perm + N;
+    int32_t* pool = aux + N;
+    uint8_t* mark = reinterpret_cast<uint8_t*>(pool + N);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ int s_M;
+
+    int M = N - 1;
+    if (MASKED) {
+        if (!online.get(w)) {
+            for (long long i = tid; i < (long long)S * R; i += kSelectThreads) idx[(size_t)w * S * R + i] = -1;
+            return;
+        }
+        if (warp == 0) {
+            int k = 0;
+            for (int v0 = 0; v0 < N; v0 += 32) {
+                const int v = v0 + lane;
+                const bool bit = (v < N) && (v != w) && online.get(v);
+                const unsigned b = __ballot_sync(0xffffffffu, bit);
+                if (bit) pool[k + __popc(b & ((1u << lane) - 1u))] = v;
+                k += __popc(b);
+            }
+            if (lane == 0) s_M = k;
+        }
+        __syncthreads();
+        M = s_M;
+    }
 
     for (int v = tid; v < N; v += kSelectThreads) mark[v] = 0;
 
@@ -55,7 +83,7 @@ k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __re
             uint64_t h = splitmix_step(hw ^ (((uint64_t)e << 32) | (uint64_t)(uint32_t)t));
             aux[t] = (int32_t)(((h >> 32) * (uint64_t)(t + 1)) >> 32);   // in [0, t]
         }
-        for (int i = tid; i < M; i += kSelectThreads) perm[i] = i + (i >= w ? 1 : 0);
+        for (int i = tid; i < M; i += kSelectThreads) perm[i] = MASKED ? pool[i] : i + (i >= w ? 1 : 0);
         __syncthreads();
         if (warp == 0) {
             if (lane == 0) {
