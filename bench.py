@@ -44,6 +44,7 @@ def parse_args():
                     help="round: the synchronization round (default); divergence: the Eq. 7 diagnostic alone")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graphs", action="store_true", help="never replay short steps from CUDA graphs")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 direct gather, 2 staged")
     ap.add_argument("--P", type=int, default=0, help="override the vector length (scaled-down runs)")
     ap.add_argument("--N", type=int, default=0, help="override the number of workers")
@@ -336,22 +337,98 @@ def main():
     sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(max(args.warmup, 0)):
         step(False)
+    torch.cuda.synchronize()
+    # A step that takes less than the CPU needs to launch it (workload 1: two kernels of a
+    # few microseconds) is replayed from CUDA graphs, one graph per buffer pair.
+    probe0 = torch.cuda.Event(enable_timing=True)
+    probe1 = torch.cuda.Event(enable_timing=True)
+    probe0.record(stream)
+    for _ in range(3):
+        step(False)
+    probe1.record(stream)
+    torch.cuda.synchronize()
+    use_graphs = (probe0.elapsed_time(probe1) / 3.0) < 0.3 and not args.no_graphs
+    graphs, agg_graphs = [], []
+    if use_graphs:
+        gs = torch.cuda.Stream()
+
+        def capture(body):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(gs):
+                body(gs)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=gs):
+                    body(gs)
+            return g
+
+        def aggregate_on(src, dst, st):
+            if wl.dtype == "bf16":
+                combo.combo_segment_aggregate_bf16(src, dst, weights, idx, wl.N, wl.P, wl.S, wl.R, stream=st)
+            elif wl.fused_sgd:
+                combo.combo_segment_aggregate_sgd(src, grads, wl.lr, dst, weights, idx, wl.N, wl.P, wl.S, wl.R,
+                                                  stream=st)
+            else:
+                combo.combo_segment_aggregate(src, dst, weights, idx, wl.N, wl.P, wl.S, wl.R, stream=st)
+
+        def whole(st, pair):
+            cur = 0
+            for t in range(wl.rounds):
+                combo.combo_select_peers(wl.sampler_seed + rank, t, wl.N, wl.S, wl.R, idx, stream=st)
+                aggregate_on(pair[cur], pair[1 - cur], st)
+                cur = 1 - cur
+
+        def only_agg(st, pair):
+            cur = 0
+            for t in range(wl.rounds):
+                aggregate_on(pair[cur], pair[1 - cur], st)
+                cur = 1 - cur
+
+        # one graph holding a step on every buffer pair (nsets steps), single-step graphs for
+        # the remainder, and the same with the aggregation launches alone
+        all_steps = capture(lambda st: [whole(st, pr) for pr in sets])
+        all_aggs = capture(lambda st: [only_agg(st, pr) for pr in sets])
+        for pair in sets:
+            graphs.append(capture(lambda st, pair=pair: whole(st, pair)))
+            agg_graphs.append(capture(lambda st, pair=pair: only_agg(st, pair)))
+        torch.cuda.synchronize()
+        all_steps.replay()
+
+        def replay_steps(big, singles):
+            for _ in range(args.steps // nsets):
+                big.replay()
+            for k in range(args.steps % nsets):
+                singles[k].replay()
     if sampler:
         sampler.wait_first_sample()
     barrier()
     t_begin = time.time()
     ev0 = torch.cuda.Event(enable_timing=True)
     ev1 = torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    for _ in range(args.steps):
-        step(True)
-    ev1.record(stream)
-    barrier()
+    if use_graphs:
+        with torch.cuda.stream(gs):
+            ev0.record(gs)
+            replay_steps(all_steps, graphs)
+            ev1.record(gs)
+            # the aggregation launches alone, same buffers, for the roofline figure
+            ga = torch.cuda.Event(enable_timing=True)
+            gb = torch.cuda.Event(enable_timing=True)
+            ga.record(gs)
+            replay_steps(all_aggs, agg_graphs)
+            gb.record(gs)
+        barrier()
+        per_launch = ga.elapsed_time(gb) / (args.steps * wl.rounds)
+        agg_events = None
+    else:
+        ev0.record(stream)
+        for _ in range(args.steps):
+            step(True)
+        ev1.record(stream)
+        barrier()
     ms_total = ev0.elapsed_time(ev1)
     t_end = time.time()
     clocks = sampler.stop(t_begin, t_end) if sampler else None
     kernel_path = combo.combo_last_kernel_path()
-    agg_ms = [a.elapsed_time(b) for a, b in agg_events]
+    agg_ms = [per_launch] if agg_events is None else [a.elapsed_time(b) for a, b in agg_events]
     combo.combo_device_status()
 
     # ---- end to end: host buffers, copies inside the timed region
@@ -428,7 +505,9 @@ def main():
                        "l2": "inputs larger than L2 (%.2f GB in + out per round)" % (pair_bytes / 1e9)
                        if nsets == 1 else "rotating over %d buffer pairs (%.0f MB) so that each step reads HBM"
                        % (nsets, nsets * pair_bytes / 1e6),
-                       "kernel_path": {1: "direct", 2: "staged"}.get(kernel_path, "?")},
+                       "kernel_path": {1: "direct", 2: "staged"}.get(kernel_path, "?"),
+                       "launch": "CUDA graph replay (step shorter than its CPU launch cost)" if use_graphs
+                       else "stream launches"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                          "kernel": "k_staged" if kernel_path == 2 else "k_direct",
