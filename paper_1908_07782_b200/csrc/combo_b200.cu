@@ -504,18 +504,26 @@ combo_status select_peers_impl(uint64_t seed, uint32_t round, int N, int S, int 
     DeviceInfo* dev = nullptr;
     combo_status rc = device_info(&dev);
     if (rc != COMBO_OK) return rc;
-    const size_t smem = combo::select_peers_smem_bytes(N);
+    // one warp per worker, up to four workers per CTA while their arrays fit
+    const size_t per_worker = (combo::select_peers_smem_bytes(N) + 15) / 16 * 16;
+    int wpb = (int)((96 * 1024) / per_worker);
+    if (wpb > combo::kSelectThreads / 32) wpb = combo::kSelectThreads / 32;
+    if (wpb < 1) wpb = 1;
+    const size_t smem = per_worker * (size_t)wpb;
+    const int blocks = (N + wpb - 1) / wpb;
     cudaError_t e = cudaSuccess;
     if (h_online) {
         if (smem > 48 * 1024)
             e = cudaFuncSetAttribute(combo::k_select_peers<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess)
-            combo::k_select_peers<true><<<N, combo::kSelectThreads, smem, st>>>(seed, round, N, S, R, idx_out, bits);
+            combo::k_select_peers<true><<<blocks, 32 * wpb, smem, st>>>(seed, round, N, S, R, idx_out, bits,
+                                                                        (int)per_worker);
     } else {
         if (smem > 48 * 1024)
             e = cudaFuncSetAttribute(combo::k_select_peers<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess)
-            combo::k_select_peers<false><<<N, combo::kSelectThreads, smem, st>>>(seed, round, N, S, R, idx_out, bits);
+            combo::k_select_peers<false><<<blocks, 32 * wpb, smem, st>>>(seed, round, N, S, R, idx_out, bits,
+                                                                         (int)per_worker);
     }
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "select_peers launch");

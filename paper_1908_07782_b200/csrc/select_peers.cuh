@@ -1,7 +1,7 @@
 // Peer selection kernel (Section 4.1 step 2, "Segments Pulling").
 //
-// One CTA per worker.  The random draw positions of a shuffle are a pure
-// function of (seed, round, worker, epoch, position), so all threads compute
+// One warp per worker.  The random draw positions of a shuffle are a pure
+// function of (seed, round, worker, epoch, position), so the lanes compute
 // them in parallel; the swaps themselves are inherently sequential and are
 // applied by one lane.  The peers of the segment being filled are kept as a
 // byte map over worker ids, which serves both the "skip what this segment
@@ -31,43 +31,40 @@ __host__ __device__ inline size_t select_peers_smem_bytes(int N) {
     return (size_t)N * 12 + (size_t)N + 16;
 }
 
-// MASKED: the pool of worker w is the ONLINE others (ascending); an offline worker issues
-// no requests and its rows are filled with -1.
+// One WARP per worker (several workers per CTA): everything is ordered by __syncwarp, no
+// CTA-wide barrier.  MASKED: the pool of worker w is the ONLINE others (ascending); an
+// offline worker issues no requests and its rows are filled with -1.
 template <bool MASKED>
 __global__ void __launch_bounds__(kSelectThreads)
 k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __restrict__ idx,
-               const WorkerBits online) {
+               const WorkerBits online, int per_worker_bytes) {
     extern __shared__ __align__(16) unsigned char sp_smem[];
-    const int w = blockIdx.x;
-    int32_t* perm = reinterpret_cast<int32_t*>(sp_smem);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int w = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (w >= N) return;
+    unsigned char* mine = sp_smem + (size_t)warp * per_worker_bytes;
+    int32_t* perm = reinterpret_cast<int32_t*>(mine);
     int32_t* aux = perm + N;
     int32_t* pool = aux + N;
     uint8_t* mark = reinterpret_cast<uint8_t*>(pool + N);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    __shared__ int s_M;
 
     int M = N - 1;
     if (MASKED) {
         if (!online.get(w)) {
-            for (long long i = tid; i < (long long)S * R; i += kSelectThreads) idx[(size_t)w * S * R + i] = -1;
+            for (long long i = lane; i < (long long)S * R; i += 32) idx[(size_t)w * S * R + i] = -1;
             return;
         }
-        if (warp == 0) {
-            int k = 0;
-            for (int v0 = 0; v0 < N; v0 += 32) {
-                const int v = v0 + lane;
-                const bool bit = (v < N) && (v != w) && online.get(v);
-                const unsigned b = __ballot_sync(0xffffffffu, bit);
-                if (bit) pool[k + __popc(b & ((1u << lane) - 1u))] = v;
-                k += __popc(b);
-            }
-            if (lane == 0) s_M = k;
+        int k = 0;
+        for (int v0 = 0; v0 < N; v0 += 32) {
+            const int v = v0 + lane;
+            const bool bit = (v < N) && (v != w) && online.get(v);
+            const unsigned b = __ballot_sync(0xffffffffu, bit);
+            if (bit) pool[k + __popc(b & ((1u << lane) - 1u))] = v;
+            k += __popc(b);
         }
-        __syncthreads();
-        M = s_M;
+        M = k;
     }
-
-    for (int v = tid; v < N; v += kSelectThreads) mark[v] = 0;
+    for (int v = lane; v < N; v += 32) mark[v] = 0;
 
     // chain: seed -> (round | worker) -> (epoch | position)
     uint64_t hw = splitmix_step(seed);
@@ -75,57 +72,55 @@ k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __re
 
     const long long total = (long long)S * (long long)R;
     const uint32_t epochs = (uint32_t)((total + M - 1) / M);
-    long long done = 0, row = 0;   // warp-0 uniform
+    long long done = 0, row = 0;   // warp-uniform
     int nc = 0;                    // peers the current segment holds so far
 
     for (uint32_t e = 0; e < epochs; ++e) {
-        for (int t = 1 + tid; t < M; t += kSelectThreads) {
+        for (int t = 1 + lane; t < M; t += 32) {
             uint64_t h = splitmix_step(hw ^ (((uint64_t)e << 32) | (uint64_t)(uint32_t)t));
             aux[t] = (int32_t)(((h >> 32) * (uint64_t)(t + 1)) >> 32);   // in [0, t]
         }
-        for (int i = tid; i < M; i += kSelectThreads) perm[i] = MASKED ? pool[i] : i + (i >= w ? 1 : 0);
-        __syncthreads();
-        if (warp == 0) {
-            if (lane == 0) {
-                for (int t = M - 1; t >= 1; --t) {          // Fisher-Yates
-                    int j = aux[t];
-                    int32_t a = perm[t]; perm[t] = perm[j]; perm[j] = a;
-                }
-                if (nc > 0) {                                // held peers go last, order kept
-                    int a = 0;
-                    for (int i = 0; i < M; ++i) if (!mark[perm[i]]) aux[a++] = perm[i];
-                    for (int i = 0; i < M; ++i) if (mark[perm[i]]) aux[a++] = perm[i];
-                    for (int i = 0; i < M; ++i) perm[i] = aux[i];
-                }
+        for (int i = lane; i < M; i += 32) perm[i] = MASKED ? pool[i] : i + (i >= w ? 1 : 0);
+        __syncwarp();
+        if (lane == 0) {
+            for (int t = M - 1; t >= 1; --t) {          // Fisher-Yates
+                int j = aux[t];
+                int32_t a = perm[t]; perm[t] = perm[j]; perm[j] = a;
             }
-            __syncwarp();
-            int pos = 0;
-            while (pos < M && done < total) {
-                int take = R - nc;
-                if (take > M - pos) take = M - pos;
-                for (int i = lane; i < take; i += 32) mark[perm[pos + i]] = 1;
-                pos += take; nc += take; done += take;
-                __syncwarp();
-                if (nc == R) {                               // emit the row ascending
-                    int32_t* out = idx + (size_t)((long long)w * S + row) * (size_t)R;
-                    int k = 0;
-                    for (int v0 = 0; v0 < N; v0 += 32) {
-                        int v = v0 + lane;
-                        bool bit = (v < N) && mark[v];
-                        unsigned b = __ballot_sync(0xffffffffu, bit);
-                        if (bit) {
-                            out[k + __popc(b & ((1u << lane) - 1u))] = v;
-                            mark[v] = 0;
-                        }
-                        k += __popc(b);
-                    }
-                    __syncwarp();
-                    nc = 0;
-                    ++row;
-                }
+            if (nc > 0) {                                // held peers go last, order kept
+                int a = 0;
+                for (int i = 0; i < M; ++i) if (!mark[perm[i]]) aux[a++] = perm[i];
+                for (int i = 0; i < M; ++i) if (mark[perm[i]]) aux[a++] = perm[i];
+                for (int i = 0; i < M; ++i) perm[i] = aux[i];
             }
         }
-        __syncthreads();
+        __syncwarp();
+        int pos = 0;
+        while (pos < M && done < total) {
+            int take = R - nc;
+            if (take > M - pos) take = M - pos;
+            for (int i = lane; i < take; i += 32) mark[perm[pos + i]] = 1;
+            pos += take; nc += take; done += take;
+            __syncwarp();
+            if (nc == R) {                               // emit the row ascending
+                int32_t* out = idx + (size_t)((long long)w * S + row) * (size_t)R;
+                int k = 0;
+                for (int v0 = 0; v0 < N; v0 += 32) {
+                    int v = v0 + lane;
+                    bool bit = (v < N) && mark[v];
+                    unsigned b = __ballot_sync(0xffffffffu, bit);
+                    if (bit) {
+                        out[k + __popc(b & ((1u << lane) - 1u))] = v;
+                        mark[v] = 0;
+                    }
+                    k += __popc(b);
+                }
+                __syncwarp();
+                nc = 0;
+                ++row;
+            }
+        }
+        __syncwarp();
     }
 }
 
