@@ -255,18 +255,6 @@ template <> struct PairStore<2, 2> {
     }
 };
 
-// Coefficients of Eq. 3 for one (worker, segment): c_j = |D_j| / sum over P_l,
-// provider order self, then peers ascending.  cf[0..R], binary32.
-__device__ __forceinline__ void eq3_coefficients(const float* __restrict__ weights,
-                                                 const int32_t* __restrict__ peers, int w, int R,
-                                                 float* cf) {
-    const float dw = weights ? weights[w] : 1.0f;
-    float den = dw;
-    for (int r = 0; r < R; ++r) den = __fadd_rn(den, weights ? weights[peers[r]] : 1.0f);
-    cf[0] = __fdiv_rn(dw, den);
-    for (int r = 0; r < R; ++r) cf[r + 1] = __fdiv_rn(weights ? weights[peers[r]] : 1.0f, den);
-}
-
 // ---------------------------------------------------------------- direct gather
 template <int EB, bool SGD>
 __device__ __forceinline__ float direct_x(const AggParams& p, int k, long long c) {
@@ -622,39 +610,39 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
 
     // Coefficient / offset table of segments l0 and l0+1, built by all consumer threads.
     auto build_table = [&](int l0_build) {
-            for (int q = ctid; q < 2 * N; q += kConsumerThreads) {
-        const int slot = q / N, w = q - slot * N;
-        const int l = l0_build + slot;
-        if (l < p.S) {
-            const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
-            float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
-            int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
-            // providers in the fixed order: the worker itself (unless it is a newcomer), then
-            // the peers ascending; a negative entry is a pull that found no online peer
-            int prov[RMAX + 1];
-            int np = 0;
-            if (!p.newcomer.get(w)) prov[np++] = w;
-            for (int r = 0; r < R; ++r) {
-                const int k = peers[r];
-                if (k >= 0) prov[np++] = k;
+        for (int q = ctid; q < 2 * N; q += kConsumerThreads) {
+            const int slot = q / N, w = q - slot * N;
+            const int l = l0_build + slot;
+            if (l < p.S) {
+                const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
+                float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
+                int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
+                // providers in the fixed order: the worker itself (unless it is a newcomer), then
+                // the peers ascending; a negative entry is a pull that found no online peer
+                int prov[RMAX + 1];
+                int np = 0;
+                if (!p.newcomer.get(w)) prov[np++] = w;
+                for (int r = 0; r < R; ++r) {
+                    const int k = peers[r];
+                    if (k >= 0) prov[np++] = k;
+                }
+                if (np == 0) prov[np++] = w;                 // nothing to aggregate: keep the own values
+                float den = p.weights ? p.weights[prov[0]] : 1.0f;
+                for (int t = 1; t < np; ++t) den = __fadd_rn(den, p.weights ? p.weights[prov[t]] : 1.0f);
+                for (int r = 0; r < np; ++r) {
+                    const int k = prov[r];
+                    cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                    // staged row of worker k: classes are stored one after another
+                    const int jk = k % p.m;
+                    int base = 0;
+                    for (int q2 = 0; q2 < jk; ++q2) base += (N - q2 + p.m - 1) / p.m;
+                    const int phase = (int)(((long long)k * p.pitch * EB) & 15);
+                    po[r] = (base + k / p.m) * p.row_bytes + phase;
+                }
+                // unused slots: coefficient zero on a row that is known to hold finite values
+                for (int r = np; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
             }
-            if (np == 0) prov[np++] = w;                 // nothing to aggregate: keep the own values
-            float den = p.weights ? p.weights[prov[0]] : 1.0f;
-            for (int t = 1; t < np; ++t) den = __fadd_rn(den, p.weights ? p.weights[prov[t]] : 1.0f);
-            for (int r = 0; r < np; ++r) {
-                const int k = prov[r];
-                cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
-                // staged row of worker k: classes are stored one after another
-                const int jk = k % p.m;
-                int base = 0;
-                for (int q2 = 0; q2 < jk; ++q2) base += (N - q2 + p.m - 1) / p.m;
-                const int phase = (int)(((long long)k * p.pitch * EB) & 15);
-                po[r] = (base + k / p.m) * p.row_bytes + phase;
-            }
-            // unused slots: coefficient zero on a row that is known to hold finite values
-            for (int r = np; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
         }
-    }
     };
     // The first tile's table does not depend on the staged data: build it while the
     // first TMA loads are in flight.
