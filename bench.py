@@ -219,6 +219,7 @@ def run_divergence(args, wl):
         combo.combo_segment_aggregate_bf16(x, out, weights, idx, wl.N, wl.P, wl.S, wl.R)
     else:
         combo.combo_segment_aggregate(x, out, weights, idx, wl.N, wl.P, wl.S, wl.R)
+    combo.combo_set_tuning(args.tile, args.stages)
     rho = torch.empty(wl.N, dtype=torch.float64, device=dev)
     scratch = torch.empty(combo.combo_divergence_scratch_bytes(wl.N) // 8, dtype=torch.float64, device=dev)
     stream = torch.cuda.current_stream()

@@ -360,8 +360,8 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
         p.coef_off = header;
         p.rowoff_off = p.coef_off + round_up((unsigned)N * 4u, 128);
         p.part_off = p.rowoff_off + round_up((unsigned)N * 4u, 128);
-        p.mean_off = p.part_off + (unsigned)combo::kConsumerThreads * V * 4u;   // G * PSTR floats at most
-        p.stage_off = p.mean_off + combo::kDivTile * 4u;
+        p.mean_off = p.part_off + 2u * combo::kConsumerThreads * V * 4u;   // two copies of G * PSTR floats
+        p.stage_off = p.mean_off + 2u * combo::kDivTile * 4u;
         p.m = m;
         const long long budget = (long long)dev->smem_optin - p.stage_off - 256;
         // tile and box: the widest of which two stages fit; with row phases one box of 256
@@ -382,8 +382,10 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
             p.row_bytes = box * EB;
             p.stage_bytes = (unsigned)(p.narr * N * p.row_bytes);
             const int fit = (int)(budget / p.stage_bytes);
+            // two tiles are in the consumers' hands at a time: three stages keep a load in flight
             int stages = (int)((112 * 1024) / p.stage_bytes);
-            if (stages < 2) stages = 2;
+            if (stages < 3) stages = 3;
+            if (t_stages >= 2) stages = t_stages;
             if (stages > combo::kMaxStages) stages = combo::kMaxStages;
             if (stages > fit) stages = fit;
             p.stages = stages;

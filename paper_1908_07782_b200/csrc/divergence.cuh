@@ -50,8 +50,8 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
     const int N = p.N, stages = p.stages;
     float* coef = reinterpret_cast<float*>(smem + p.coef_off);     // c_j = |D_j| / sum |D|
     int* rowoff = reinterpret_cast<int*>(smem + p.rowoff_off);     // staged byte offset of worker j's tile part
-    float* part = reinterpret_cast<float*>(smem + p.part_off);     // [G][PSTR]
-    float* mean = reinterpret_cast<float*>(smem + p.mean_off);     // [TC]
+    float* part = reinterpret_cast<float*>(smem + p.part_off);     // [2][G][PSTR]
+    float* mean = reinterpret_cast<float*>(smem + p.mean_off);     // [2][kDivTile]
     const int block_bytes = N * p.row_bytes;
 
     if (tid == 0) {
@@ -131,61 +131,100 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
         }
     };
 
-    long long n = 0;
-    for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
-        const int s = (int)(n % stages);
-        const uint32_t ph = (uint32_t)((n / stages) & 1);
-        if (!mbar_wait(smem_u32(&hdr->full[s]), ph)) { staged_fail(13); return; }
-        const unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
-        const unsigned char* xsrc = stage + (p.narr - 1) * block_bytes;     // rows the mean is taken over
-
-        // (A) weighted column sums of this thread's row group; columns past the end of the
-        // rows were zero-filled by the TMA unit and contribute nothing anywhere below
-        if (au < NU) {
-            float a[EPU];
+    // EPU consecutive floats of shared memory as one vector access (16-byte aligned groups)
+    auto store_floats = [](float* q, const float (&v)[EPU]) {
+        if constexpr (EPU % 4 == 0) {
 #pragma unroll
-            for (int i = 0; i < EPU; ++i) a[i] = 0.0f;
-            for (int j = ag; j < N; j += G) {
-                float x[EPU];
-                load_unit(xsrc + rowoff[j] + au * UB, x);
-                const float c = coef[j];
+            for (int e = 0; e < EPU; e += 4) *reinterpret_cast<float4*>(q + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+        } else if constexpr (EPU == 2) {
+            *reinterpret_cast<float2*>(q) = make_float2(v[0], v[1]);
+        } else {
+            q[0] = v[0];
+        }
+    };
+    auto load_floats = [](const float* q, float (&v)[EPU]) {
+        if constexpr (EPU % 4 == 0) {
 #pragma unroll
-                for (int i = 0; i < EPU; ++i) a[i] = fmaf(c, x[i], a[i]);
+            for (int e = 0; e < EPU; e += 4) {
+                const float4 t = *reinterpret_cast<const float4*>(q + e);
+                v[e] = t.x; v[e + 1] = t.y; v[e + 2] = t.z; v[e + 3] = t.w;
             }
+        } else if constexpr (EPU == 2) {
+            const float2 t = *reinterpret_cast<const float2*>(q);
+            v[0] = t.x; v[1] = t.y;
+        } else {
+            v[0] = q[0];
+        }
+    };
+
+    // Software pipeline over this CTA's tiles, one consumer-wide barrier per tile:
+    //   step i:  (A) partial column sums of tile i      -> part[i & 1]
+    //            barrier
+    //            (A2) column means of tile i            -> mean[i & 1]
+    //            (B) squared deviations of tile i-1 against mean[(i-1) & 1], stage released
+    // The barrier of step i orders A2(i-1) before B(i-1) and B(i-2) before A2(i); the two
+    // copies of `part` and `mean` keep neighbouring steps off each other's data.
+    const long long n_my = (p.n_tiles > (long long)blockIdx.x)
+                               ? (p.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    for (long long i = 0; i <= n_my; ++i) {
+        if (i < n_my) {
+            const int s = (int)(i % stages);
+            if (!mbar_wait(smem_u32(&hdr->full[s]), (uint32_t)((i / stages) & 1))) { staged_fail(13); return; }
+            const unsigned char* xsrc = smem + p.stage_off + (size_t)s * p.stage_bytes + (p.narr - 1) * block_bytes;
+            float* pt = part + (i & 1) * (G * PSTR);
+            // (A) weighted column sums of this thread's row group; columns past the end of the
+            // rows were zero-filled by the TMA unit and contribute nothing anywhere below
+            if (au < NU) {
+                float a[EPU];
 #pragma unroll
-            for (int i = 0; i < EPU; ++i) part[ag * PSTR + au * EPU + i] = a[i];
+                for (int e = 0; e < EPU; ++e) a[e] = 0.0f;
+                for (int j = ag; j < N; j += G) {
+                    float x[EPU];
+                    load_unit(xsrc + rowoff[j] + au * UB, x);
+                    const float c = coef[j];
+#pragma unroll
+                    for (int e = 0; e < EPU; ++e) a[e] = fmaf(c, x[e], a[e]);
+                }
+                store_floats(pt + ag * PSTR + au * EPU, a);
+            }
         }
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(14); return; }
-        if (ctid < TC) {
+        if (i < n_my && ctid < TC) {
+            const float* pt = part + (i & 1) * (G * PSTR);
             float m = 0.0f;
 #pragma unroll
-            for (int g = 0; g < G; ++g) m = __fadd_rn(m, part[g * PSTR + ctid]);
-            mean[ctid] = m;
+            for (int g = 0; g < G; ++g) m = __fadd_rn(m, pt[g * PSTR + ctid]);
+            mean[(i & 1) * kDivTile + ctid] = m;
         }
-        if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(15); return; }
-
-        // (B) warp per row: squared deviations of the workers' own models
+        if (i >= 1) {
+            // (B) warp per row: squared deviations of the workers' own models, tile i-1
+            const long long t = i - 1;
+            const int s = (int)(t % stages);
+            const unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
+            const float* mn = mean + (t & 1) * kDivTile;
 #pragma unroll
-        for (int sl = 0; sl < kDivSlots; ++sl) {
-            const int i = cw + sl * kConsumerWarps;
-            if (i < N) {
-                float ssum = 0.0f;
-                const unsigned char* row = stage + rowoff[i];
+            for (int sl = 0; sl < kDivSlots; ++sl) {
+                const int r = cw + sl * kConsumerWarps;
+                if (r < N) {
+                    float ssum = 0.0f;
+                    const unsigned char* row = stage + rowoff[r];
 #pragma unroll
-                for (int u = lane; u < NU; u += 32) {
-                    float x[EPU];
-                    load_unit(row + u * UB, x);
+                    for (int u = lane; u < NU; u += 32) {
+                        float x[EPU], mu[EPU];
+                        load_unit(row + u * UB, x);
+                        load_floats(mn + u * EPU, mu);
 #pragma unroll
-                    for (int e = 0; e < EPU; ++e) {
-                        const float d = __fsub_rn(x[e], mean[u * EPU + e]);
-                        ssum = fmaf(d, d, ssum);
+                        for (int e = 0; e < EPU; ++e) {
+                            const float d = __fsub_rn(x[e], mu[e]);
+                            ssum = fmaf(d, d, ssum);
+                        }
                     }
+                    acc[sl] += (double)ssum;
                 }
-                acc[sl] += (double)ssum;
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
     }
     // per-CTA partial sums: one entry per row, written by the warp that owns the row
 #pragma unroll

@@ -452,11 +452,27 @@ struct StagedHeader {
 
 __device__ __forceinline__ void staged_fail(int code) { atomicCAS(&g_dev_status, 0, code); }
 
+// Bounded wait that never lets the warp be suspended for long: for barriers between
+// consumer warps, which complete within a fraction of a microsecond.
+__device__ __forceinline__ bool mbar_wait_brisk(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+#pragma unroll 1
+    for (uint32_t it = 0; it < (kWaitCap << 3); ++it) {
+        asm volatile(
+            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
 // Consumer-wide barrier with a bounded wait (all 16 consumer warps).
 __device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t& phase, int lane) {
     __syncwarp();
     if (lane == 0) mbar_arrive(bar);
-    bool ok = mbar_wait(bar, phase & 1u);
+    bool ok = mbar_wait_brisk(bar, phase & 1u);
     phase ^= 1u;
     return ok;
 }
