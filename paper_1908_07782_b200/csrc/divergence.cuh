@@ -35,7 +35,7 @@ struct DivParams {
 // which two stages fit), threads work on 128-bit vectors.  WORD: rows whose pitch is only a
 // multiple of 4 bytes are staged per row class with their phase (see the aggregation
 // kernel), TC = 256 - 16/e, and threads work on 4-byte words at the row's phase.
-template <int EB, int TC, bool WORD>
+template <int EB, int TC, bool WORD, bool PIPE = !WORD>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
     constexpr int UB = WORD ? 4 : 16;                  // bytes a thread takes at a time
@@ -196,9 +196,13 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
             for (int g = 0; g < G; ++g) m = __fadd_rn(m, pt[g * PSTR + ctid]);
             mean[(i & 1) * kDivTile + ctid] = m;
         }
-        if (i >= 1) {
-            // (B) warp per row: squared deviations of the workers' own models, tile i-1
-            const long long t = i - 1;
+        if (!PIPE) {
+            // unpipelined form: the means of tile i must be complete before its deviations
+            if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(15); return; }
+        }
+        if (PIPE ? (i >= 1) : (i < n_my)) {
+            // (B) warp per row: squared deviations of the workers' own models, tile i-1 (i when unpipelined)
+            const long long t = PIPE ? i - 1 : i;
             const int s = (int)(t % stages);
             const unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
             const float* mn = mean + (t & 1) * kDivTile;
