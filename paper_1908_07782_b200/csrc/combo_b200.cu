@@ -64,6 +64,29 @@ inline bool overlaps(const void* a, const void* b, size_t bytes) {
 
 inline unsigned round_up(unsigned v, unsigned q) { return (v + q - 1) / q * q; }
 
+// ---------------------------------------------------------------- tile dispensers
+// Launches of the staged kernel take the slots of combo::g_tile_slots in turn.  A slot is
+// zero when idle (the kernel's last CTA resets it), so launches that overlap on the device
+// only need different slots: 256 of them cover any number of kernels that can be resident.
+combo::TileSlot* g_slot_base[64];
+unsigned g_slot_seq = 0;
+
+combo_status next_tile_slot(combo::TileSlot** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return COMBO_ERR_UNSUPPORTED;
+    if (!g_slot_base[dev]) {
+        combo::TileSlot* ptr = nullptr;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), combo::g_tile_slots);
+        if (e != cudaSuccess || !ptr) return cuda_fail(e, "cudaGetSymbolAddress(tile slots)");
+        g_slot_base[dev] = ptr;
+    }
+    const unsigned seq = __atomic_fetch_add(&g_slot_seq, 1u, __ATOMIC_RELAXED);
+    *out = g_slot_base[dev] + (seq % combo::kTileSlots);
+    return COMBO_OK;
+}
+
 // ---------------------------------------------------------------- staged plan
 struct StagedPlan {
     bool ok;
@@ -304,6 +327,8 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
         combo::TileMaps maps;
         StagedPlan plan = plan_staged(p, maps, EB, sgd, *dev);
         if (plan.ok) {
+            rc = next_tile_slot(&p.sched);
+            if (rc != COMBO_OK) return rc;
             cudaError_t e = launch_staged(p, maps, plan, EB, sgd, st);
             if (e != cudaSuccess) return cuda_fail(e, "staged aggregation launch");
             t_last_path = 2;

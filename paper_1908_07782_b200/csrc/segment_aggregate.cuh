@@ -49,6 +49,17 @@ constexpr int kMaxBoxes = 8;              // x-boxes per tile
 constexpr uint32_t kWaitCap = 1u << 23;   // polls before a wait is declared dead
 constexpr uint32_t kWaitHintNs = 1000;    // time a single poll may stay suspended
 
+// Tile dispenser of one launch (global memory owned by the library, one of a ring of
+// slots).  `next` hands out tiles beyond the first one of each CTA; the last CTA to leave
+// puts the slot back to zero, so a slot is clean whenever a launch picks it up.
+struct TileSlot {
+    unsigned long long next;
+    unsigned int done;
+    unsigned int pad;
+};
+constexpr int kTileSlots = 256;
+__device__ TileSlot g_tile_slots[kTileSlots];
+
 // One flag per worker (up to COMBO_MAX_WORKERS), passed by value (Section 4.2: online /
 // offline workers, newcomers).
 struct WorkerBits {
@@ -78,6 +89,7 @@ struct AggParams {
     unsigned tab_off;    // byte offset of the coefficient table in shared memory
     unsigned stage_off;  // byte offset of stage 0
     unsigned stage_bytes;
+    TileSlot* sched;     // tile dispenser of this launch
     WorkerBits newcomer; // workers that aggregate without their own model (Section 4.2)
 };
 
@@ -436,10 +448,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 }
 
 struct TileMeta {
+    long long tile;  // tile held by the stage, or -1: no more work
     long long bnd;   // local column where segment l0+1 starts
     int l0;          // segment of the tile's first column
     int pad;
 };
+
 
 // shared-memory header: barriers and per-stage metadata
 struct StagedHeader {
@@ -568,24 +582,39 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         if (issuer) asm volatile("prefetch.tensormap [%0];" ::"l"(my_map) : "memory");
         const uint32_t my_dst_off = (uint32_t)((a * p.nbx + b) * block_bytes + class_base * p.row_bytes);
         const int tile_cols_per_box = p.T / p.nbx;
+        // Tiles are handed out dynamically: SMs differ by some 10 % in the HBM bandwidth they
+        // get, and with a fixed share of tiles the slowest CTA would set the kernel time.  Each
+        // CTA starts on tile blockIdx.x; every further tile comes from the launch's counter.
         long long n = 0;
-        for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
+        long long tile = blockIdx.x;
+        for (;; ++n) {
             const int s = (int)(n % stages);
             const uint32_t ph = (uint32_t)((n / stages) & 1);
             if (!mbar_wait_patient(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); break; }
             const long long t0 = tile * (long long)p.T;
             const uint32_t bar = smem_u32(&hdr->full[s]);
+            const bool last = tile >= p.n_tiles;
             if (lane == 0) {
                 TileMeta& mt = hdr->meta[s];
-                const int l0 = (int)((p.p_begin + t0) / p.L);
-                mt.l0 = l0;
-                mt.bnd = (long long)(l0 + 1) * p.L - p.p_begin;
-                mbar_arrive_expect_tx(bar, p.stage_bytes);
+                if (last) {
+                    mt.tile = -1;                                  // tells the consumers to leave
+                    mbar_arrive(bar);
+                } else {
+                    const int l0 = (int)((p.p_begin + t0) / p.L);
+                    mt.tile = tile;
+                    mt.l0 = l0;
+                    mt.bnd = (long long)(l0 + 1) * p.L - p.p_begin;
+                    mbar_arrive_expect_tx(bar, p.stage_bytes);
+                }
             }
             __syncwarp();
+            if (last) { ++n; break; }
             if (issuer)
                 tma_load_2d(smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) + my_dst_off, my_map,
                             (int)(t0 + (long long)b * tile_cols_per_box), 0, bar);
+            unsigned long long got = 0;
+            if (lane == 0) got = atomicAdd(&p.sched->next, 1ULL);
+            tile = (long long)gridDim.x + (long long)__shfl_sync(0xffffffffu, got, 0);
         }
         // Leave last: every stage this warp armed must have landed before the CTA's
         // shared memory can be released, even if the consumers gave up.
@@ -594,6 +623,13 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             for (long long q = first; q < n; ++q) {
                 const int s = (int)(q % stages);
                 if (!mbar_wait(smem_u32(&hdr->full[s]), (uint32_t)((q / stages) & 1))) staged_fail(2);
+            }
+            // the last CTA to get here leaves the dispenser clean for the next launch that uses it
+            __threadfence();
+            if (atomicAdd(&p.sched->done, 1u) == gridDim.x - 1) {
+                p.sched->next = 0;
+                p.sched->done = 0;
+                __threadfence();
             }
         }
         return;
@@ -668,11 +704,12 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(7); return; }
     }
 
-    long long n = 0;
-    for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
+    for (long long n = 0;; ++n) {
         const int s = (int)(n % stages);
         const uint32_t ph = (uint32_t)((n / stages) & 1);
         if (!mbar_wait(smem_u32(&hdr->full[s]), ph)) { staged_fail(3); return; }
+        const long long tile = hdr->meta[s].tile;
+        if (tile < 0) break;
         const long long m_bnd = hdr->meta[s].bnd;
         const int m_l0 = hdr->meta[s].l0;
         unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
