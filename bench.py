@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--rounds", type=int, default=0, help="override the rounds per step")
     ap.add_argument("--tile", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="ordinary launches instead of programmatic stream serialization")
     return ap.parse_args()
 
 
@@ -282,6 +284,7 @@ def main():
     combo.load()
     combo.combo_set_kernel_path(args.path)
     combo.combo_set_tuning(args.tile, args.stages)
+    combo.combo_set_launch_overlap(not args.no_overlap)
 
     # every rank: an independent replica of the workload (seed offset by rank)
     seed = 1000 * rank

@@ -275,6 +275,15 @@ void combo_set_kernel_path(int path);
  * the call fall back to the direct kernel. */
 void combo_set_tuning(int tile_elems, int stages);
 
+/* This thread only: whether the staged aggregation kernel is launched with
+ * programmatic stream serialization (default 1).  With it the kernel may be
+ * scheduled while the preceding kernel of the same stream is still draining;
+ * it waits for that kernel to complete before its first access to global
+ * memory, so stream order as seen through memory is unchanged.  What it
+ * hides is launch latency and set-up between back-to-back rounds (Section
+ * 4.1: one synchronization per iteration).  0 = ordinary launches. */
+void combo_set_launch_overlap(int on);
+
 const char* combo_status_string(combo_status status);
 const char* combo_last_cuda_error(void);
 int combo_version(void);

@@ -6,5 +6,6 @@ from .binding import (ComboError, combo_aggregation_divergence, combo_aggregatio
                       combo_segment_aggregate_bf16, combo_segment_aggregate_cols,
                       combo_segment_aggregate_members, combo_segment_aggregate_sgd, combo_select_peers,
                       combo_select_peers_online,
-                      combo_select_peers_default_stream, combo_set_kernel_path, combo_set_tuning,
+                      combo_select_peers_default_stream, combo_set_kernel_path, combo_set_launch_overlap,
+                      combo_set_tuning,
                       combo_validate_idx, combo_version, load)

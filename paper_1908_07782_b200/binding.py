@@ -67,6 +67,8 @@ def load():
     lib.combo_set_kernel_path.restype = None
     lib.combo_set_tuning.argtypes = [i32, i32]
     lib.combo_set_tuning.restype = None
+    lib.combo_set_launch_overlap.argtypes = [i32]
+    lib.combo_set_launch_overlap.restype = None
     lib.combo_status_string.argtypes = [i32]
     lib.combo_status_string.restype = ctypes.c_char_p
     lib.combo_last_cuda_error.argtypes = []
@@ -218,6 +220,10 @@ def combo_set_kernel_path(path: int) -> None:
 
 def combo_set_tuning(tile_elems: int = 0, stages: int = 0) -> None:
     load().combo_set_tuning(tile_elems, stages)
+
+
+def combo_set_launch_overlap(on: bool = True) -> None:
+    load().combo_set_launch_overlap(1 if on else 0)
 
 
 def combo_version() -> int:

@@ -21,6 +21,7 @@ thread_local int t_last_path = 0;
 thread_local int t_force_path = 0;
 thread_local int t_tile = 0;
 thread_local int t_stages = 0;
+thread_local int t_overlap = 1;
 
 struct DeviceInfo {
     int known;       // 0 unknown, 1 supported, -1 unsupported
@@ -231,8 +232,21 @@ cudaError_t launch_staged_inst(const AggParams& p, const combo::TileMaps& maps, 
     auto kern = combo::k_staged<EB, GB, SGD, RT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem);
     if (e != cudaSuccess) return e;
-    kern<<<plan.grid, combo::kStagedThreads, plan.smem, st>>>(p, maps);
-    return cudaGetLastError();
+    // Programmatic stream serialization: the kernel may be scheduled while the preceding
+    // kernel of the stream drains (it waits for that kernel's completion itself, before its
+    // first global access), which hides launch latency and set-up between back-to-back rounds.
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)plan.grid);
+    cfg.blockDim = dim3((unsigned)combo::kStagedThreads);
+    cfg.dynamicSmemBytes = plan.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = t_overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, p, maps);
 }
 
 template <int EB, int GB, bool SGD>
@@ -756,6 +770,8 @@ void combo_set_tuning(int tile_elems, int stages) {
     t_tile = tile_elems > 0 ? tile_elems : 0;
     t_stages = stages > 0 ? stages : 0;
 }
+
+void combo_set_launch_overlap(int on) { t_overlap = on ? 1 : 0; }
 
 const char* combo_status_string(combo_status status) {
     switch (status) {

@@ -568,6 +568,13 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // When launched with programmatic stream serialization this CTA may have started while
+    // the preceding kernel of the stream was still draining: everything above touched only
+    // this CTA's shared memory.  From here on global memory is read and written, so wait for
+    // that kernel to have completed, then let the next launch of the stream start its own
+    // set-up as SMs become free.  (Both are no-ops in an ordinary launch.)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -584,12 +591,19 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         const int tile_cols_per_box = p.T / p.nbx;
         // Tiles are handed out dynamically: SMs differ by some 10 % in the HBM bandwidth they
         // get, and with a fixed share of tiles the slowest CTA would set the kernel time.  Each
-        // CTA starts on tile blockIdx.x; every further tile comes from the launch's counter.
+        // The first ring of tiles is fixed (tile blockIdx.x + i * gridDim.x fills stage i), so
+        // that the pipeline fills without waiting for anything; every further tile comes from
+        // the launch's counter.  The counter is asked one tile ahead, before the wait for a
+        // free stage, which hides the round trip of the atomic (about a microsecond).
         long long n = 0;
         long long tile = blockIdx.x;
+        const long long n_static = (long long)stages * gridDim.x;
         for (;; ++n) {
             const int s = (int)(n % stages);
             const uint32_t ph = (uint32_t)((n / stages) & 1);
+            const bool ask = n + 1 >= stages && tile < p.n_tiles;
+            unsigned long long got = 0;
+            if (ask && lane == 0) got = atomicAdd(&p.sched->next, 1ULL);
             if (!mbar_wait_patient(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); break; }
             const long long t0 = tile * (long long)p.T;
             const uint32_t bar = smem_u32(&hdr->full[s]);
@@ -612,9 +626,8 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             if (issuer)
                 tma_load_2d(smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) + my_dst_off, my_map,
                             (int)(t0 + (long long)b * tile_cols_per_box), 0, bar);
-            unsigned long long got = 0;
-            if (lane == 0) got = atomicAdd(&p.sched->next, 1ULL);
-            tile = (long long)gridDim.x + (long long)__shfl_sync(0xffffffffu, got, 0);
+            tile = ask ? n_static + (long long)__shfl_sync(0xffffffffu, got, 0)
+                       : (long long)blockIdx.x + (n + 1) * (long long)gridDim.x;
         }
         // Leave last: every stage this warp armed must have landed before the CTA's
         // shared memory can be released, even if the consumers gave up.
