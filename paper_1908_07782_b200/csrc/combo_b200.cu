@@ -158,7 +158,11 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     plan.rt = (p.R >= 1 && p.R <= 4 && (plan.gb == 16 || (EB == 2 && plan.gb == 4))) ? p.R : -1;
     const int rmax = plan.rt >= 0 ? plan.rt : combo::kStagedMaxR;
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
-    const unsigned table = round_up(2u * p.N * (unsigned)combo::table_entry_bytes(rmax), 128);
+    // the coefficient table holds every segment when that is small (no rebuilds on the way,
+    // which matters for short kernels), else two segments at a time
+    const unsigned entry = (unsigned)combo::table_entry_bytes(rmax);
+    const int tab_slots = ((unsigned long long)p.S * p.N * entry <= 24u * 1024u && p.S >= 2) ? p.S : 2;
+    const unsigned table = round_up((unsigned)tab_slots * p.N * entry, 128);
     const long long budget = (long long)dev.smem_optin - header - table - 256;
 
     // candidate tiles: (T, box_w, nbx)
@@ -212,6 +216,7 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     p.row_bytes = c.box_w * EB;
     p.stage_bytes = (unsigned)stage_bytes(c);
     p.tab_off = header;
+    p.tab_slots = tab_slots;
     p.stage_off = header + table;
     p.n_tiles = tiles(c);
     for (int a = 0; a < narr; ++a)

@@ -87,6 +87,7 @@ struct AggParams {
     int stages;
     int row_bytes;       // shared-memory bytes per staged row of one box = box_w * e
     unsigned tab_off;    // byte offset of the coefficient table in shared memory
+    int tab_slots;       // segments the table holds: all S of them, or 2 (rebuilt on the way)
     unsigned stage_off;  // byte offset of stage 0
     unsigned stage_bytes;
     TileSlot* sched;     // tile dispenser of this launch
@@ -263,6 +264,44 @@ template <> struct PairStore<2, 2> {
             const uint32_t w = pack_bf16x2_rn(pair_lo(a[i]), pair_hi(a[i]));
             if (mask >> (2 * i) & 1u) __stcs(reinterpret_cast<unsigned short*>(p + (2 * i) * 64), (unsigned short)(w & 0xffffu));
             if (mask >> (2 * i + 1) & 1u) __stcs(reinterpret_cast<unsigned short*>(p + (2 * i + 1) * 64), (unsigned short)(w >> 16));
+        }
+    }
+};
+
+// Word-mode stores of a whole box: every piece lies inside the row except, for the lanes
+// with `last_on` false, the last piece of the box's last 512-byte item (the box holds
+// 16 bytes less than a whole number of items).
+template <int EB, int GB> struct PairStoreBox;
+template <> struct PairStoreBox<4, 4> {
+    template <bool LAST>
+    __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[2], bool last_on) {
+        __stcs(reinterpret_cast<uint32_t*>(p), (uint32_t)a[0]);
+        __stcs(reinterpret_cast<uint32_t*>(p + 128), (uint32_t)(a[0] >> 32));
+        __stcs(reinterpret_cast<uint32_t*>(p + 256), (uint32_t)a[1]);
+        if (LAST) stcs_b32_if(p + 384, (uint32_t)(a[1] >> 32), last_on);
+        else __stcs(reinterpret_cast<uint32_t*>(p + 384), (uint32_t)(a[1] >> 32));
+    }
+};
+template <> struct PairStoreBox<2, 4> {
+    template <bool LAST>
+    __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[4], bool last_on) {
+#pragma unroll
+        for (int i = 0; i < 3; ++i)
+            __stcs(reinterpret_cast<uint32_t*>(p + i * 128), pack_bf16x2_rn(pair_lo(a[i]), pair_hi(a[i])));
+        const uint32_t w3 = pack_bf16x2_rn(pair_lo(a[3]), pair_hi(a[3]));
+        if (LAST) stcs_b32_if(p + 384, w3, last_on);             // predicated, no branch
+        else __stcs(reinterpret_cast<uint32_t*>(p + 384), w3);
+    }
+};
+template <> struct PairStoreBox<2, 2> {
+    template <bool LAST>
+    __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[4], bool last_on) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t w = pack_bf16x2_rn(pair_lo(a[i]), pair_hi(a[i]));
+            __stcs(reinterpret_cast<unsigned short*>(p + (2 * i) * 64), (unsigned short)(w & 0xffffu));
+            if (i < 3 || !LAST || last_on)
+                __stcs(reinterpret_cast<unsigned short*>(p + (2 * i + 1) * 64), (unsigned short)(w >> 16));
         }
     }
 };
@@ -541,6 +580,26 @@ __device__ __forceinline__ void item_fast(uint32_t base, const RowCtx<RMAX>& c, 
     PairStore<EB, GB>::run(outp, acc, mask);
 }
 
+// The same for a lane's share of an item of a whole word-mode box (see PairStoreBox).
+template <int EB, int GB, int RMAX, bool FIXED_R, bool LAST>
+__device__ __forceinline__ void item_box(uint32_t base, const RowCtx<RMAX>& c, int R, unsigned char* outp,
+                                         bool last_on) {
+    constexpr int NP = ElemOps<EB>::V / 2;
+    f32x2 acc[NP], x[NP];
+    PairLoad<EB, GB>::run(base + c.poff[0], x);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) acc[i] = mul2(c.c2[0], x[i]);
+#pragma unroll
+    for (int r = 1; r <= RMAX; ++r) {
+        if (FIXED_R || r <= R) {
+            PairLoad<EB, GB>::run(base + c.poff[r], x);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) acc[i] = fma2(c.c2[r], x[i], acc[i]);
+        }
+    }
+    PairStoreBox<EB, GB>::template run<LAST>(outp, acc, last_on);
+}
+
 template <int EB, int GB, bool SGD, int RT>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
@@ -556,7 +615,8 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     const int N = p.N, R = (RT >= 0) ? RT : p.R;
     const int stages = p.stages;
     const int narr = SGD ? 2 : 1;
-    unsigned char* tab = smem + p.tab_off;                 // [2][N] entries of ENT bytes
+    unsigned char* tab = smem + p.tab_off;                 // [tab_slots][N] entries of ENT bytes
+    const bool whole_table = p.tab_slots >= p.S;           // every segment has its slot: never rebuilt
     const int block_bytes = N * p.row_bytes;               // one x-box of all rows
 
     if (tid == 0) {
@@ -573,8 +633,10 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     // this CTA's shared memory.  From here on global memory is read and written, so wait for
     // that kernel to have completed, then let the next launch of the stream start its own
     // set-up as SMs become free.  (Both are no-ops in an ordinary launch.)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    auto wait_for_preceding_kernel = [] {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -586,7 +648,8 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         int class_base = 0;                                 // staged row index of the class's first row
         for (int q = 0; q < j; ++q) class_base += (N - q + p.m - 1) / p.m;
         const CUtensorMap* my_map = &maps.map[issuer ? a : 0][issuer ? j : 0];
-        if (issuer) asm volatile("prefetch.tensormap [%0];" ::"l"(my_map) : "memory");
+        if (issuer) asm volatile("prefetch.tensormap [%0];" ::"l"(my_map) : "memory");   // a kernel parameter
+        wait_for_preceding_kernel();
         const uint32_t my_dst_off = (uint32_t)((a * p.nbx + b) * block_bytes + class_base * p.row_bytes);
         const int tile_cols_per_box = p.T / p.nbx;
         // Tiles are handed out dynamically: SMs differ by some 10 % in the HBM bandwidth they
@@ -649,6 +712,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     }
 
     // ---------------------------------------------------------------- consumers
+    wait_for_preceding_kernel();
     const int cw = warp - 1;
     const int ctid = tid - 32;
     uint32_t csync_phase = 0;
@@ -674,8 +738,8 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     }
 
     // Coefficient / offset table of segments l0 and l0+1, built by all consumer threads.
-    auto build_table = [&](int l0_build) {
-        for (int q = ctid; q < 2 * N; q += kConsumerThreads) {
+    auto build_table = [&](int l0_build, int nslots) {
+        for (int q = ctid; q < nslots * N; q += kConsumerThreads) {
             const int slot = q / N, w = q - slot * N;
             const int l = l0_build + slot;
             if (l < p.S) {
@@ -712,8 +776,12 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     // The first tile's table does not depend on the staged data: build it while the
     // first TMA loads are in flight.
     if ((long long)blockIdx.x < p.n_tiles) {
-        cached_l0 = (int)((p.p_begin + (long long)blockIdx.x * p.T) / p.L);
-        build_table(cached_l0);
+        if (whole_table) {
+            build_table(0, p.S);
+        } else {
+            cached_l0 = (int)((p.p_begin + (long long)blockIdx.x * p.T) / p.L);
+            build_table(cached_l0, 2);
+        }
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(7); return; }
     }
 
@@ -727,11 +795,13 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         const int m_l0 = hdr->meta[s].l0;
         unsigned char* stage = smem + p.stage_off + (size_t)s * p.stage_bytes;
         const uint32_t stage_s = smem_u32(stage);
+        // entries of segment l0 (those of l0 + 1 follow them)
+        const unsigned char* tab0 = whole_table ? tab + (size_t)m_l0 * N * ENT : tab;
 
-        if (m_l0 != cached_l0) {
+        if (!whole_table && m_l0 != cached_l0) {
             // table for segments l0 and l0+1 (rebuilt at most S times per CTA)
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(4); return; }
-            build_table(m_l0);
+            build_table(m_l0, 2);
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
             cached_l0 = m_l0;
         }
@@ -757,11 +827,32 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         const bool interior = (m_bnd >= t1) && (t0 + p.T <= p.width);   // one segment, whole tile
 
         int row = row_begin, xb = xb_begin;
-        if (interior) {
+        if (GB < 16 && interior) {
+            // word mode: the tile is one box, a unit is a whole row of it, and only the last
+            // piece of a row can lie outside the payload (a loop-invariant lane predicate)
+            if constexpr (GB < 16) {
+                RowCtx<RMAX> c;
+                const unsigned char* ent = tab0 + (size_t)u_begin * ENT;
+                unsigned char* orow = p.out + (size_t)u_begin * pitch_bytes + (size_t)t0 * EB + lane * GB;
+                const uint32_t lane_base = stage_s + lane * GB;
+                const bool last_on = (CPB - 1) * 512 + lane * GB + (PIECES - 1) * PSTRIDE < box_payload;
+#pragma unroll 2
+                for (int u = u_begin; u < u_end; ++u) {
+                    load_entry<RMAX>(ent, c);
+#pragma unroll
+                    for (int ch = 0; ch < CPB - 1; ++ch)
+                        item_box<EB, GB, RMAX, (RT >= 0), false>(lane_base + ch * 512, c, R, orow + ch * 512, true);
+                    item_box<EB, GB, RMAX, (RT >= 0), true>(lane_base + (CPB - 1) * 512, c, R,
+                                                            orow + (CPB - 1) * 512, last_on);
+                    ent += ENT;
+                    orow += pitch_bytes;
+                }
+            }
+        } else if (interior) {
             // every unit is whole and lies in segment l0: the lean loop, rows outside, boxes inside
             RowCtx<RMAX> c;
             const int nbx = p.nbx;
-            const unsigned char* ent = tab + (size_t)row * ENT;
+            const unsigned char* ent = tab0 + (size_t)row * ENT;
             unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
             const uint32_t lane_base = stage_s + lane * GB;
             int u = u_begin;
@@ -794,7 +885,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                         const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
                         if (whole && one_seg) {
                             RowCtx<RMAX> cc;
-                            load_entry<RMAX>(tab + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
+                            load_entry<RMAX>(tab0 + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
                             item_fast<EB, GB, RMAX, (RT >= 0)>(
                                 ubase, cc, R, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
                             done = true;
@@ -809,7 +900,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                             for (int e = 0; e < EPP; ++e) {
                                 const long long col = t0 + (xb * box_payload + pin) / EB + e;
                                 if (col >= p.width) continue;
-                                const unsigned char* ent = tab + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
+                                const unsigned char* ent = tab0 + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
                                 const float* cf = reinterpret_cast<const float*>(ent);       // pairs
                                 const int* po = reinterpret_cast<const int*>(cf + 2 * (RMAX + 1));
                                 const unsigned char* eb = stage + xb * block_bytes + pin + e * EB;
