@@ -560,20 +560,23 @@ combo_status select_peers_impl(uint64_t seed, uint32_t round, int N, int S, int 
     const size_t smem = per_worker * (size_t)wpb;
     const int blocks = (N + wpb - 1) / wpb;
     cudaError_t e = cudaSuccess;
-    if (h_online) {
-        if (smem > 48 * 1024)
-            e = cudaFuncSetAttribute(combo::k_select_peers<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess)
-            combo::k_select_peers<true><<<blocks, 32 * wpb, smem, st>>>(seed, round, N, S, R, idx_out, bits,
-                                                                        (int)per_worker);
-    } else {
-        if (smem > 48 * 1024)
-            e = cudaFuncSetAttribute(combo::k_select_peers<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess)
-            combo::k_select_peers<false><<<blocks, 32 * wpb, smem, st>>>(seed, round, N, S, R, idx_out, bits,
-                                                                         (int)per_worker);
+    auto kern = h_online ? combo::k_select_peers<true> : combo::k_select_peers<false>;
+    if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) {
+        // may start under the preceding kernel of the stream (it waits before its first write)
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3((unsigned)blocks);
+        cfg.blockDim = dim3(32u * (unsigned)wpb);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = t_overlap ? 1 : 0;
+        e = cudaLaunchKernelEx(&cfg, kern, seed, round, N, S, R, idx_out, bits, (int)per_worker);
     }
-    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "select_peers launch");
     return COMBO_OK;
 }

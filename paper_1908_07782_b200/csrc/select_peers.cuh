@@ -6,6 +6,12 @@
 // applied by one lane.  The peers of the segment being filled are kept as a
 // byte map over worker ids, which serves both the "skip what this segment
 // already holds" rule after a refill and the ascending output order.
+//
+// Section 4.1 notes that the pull requests can be sent before the local update has
+// finished, since they do not depend on it.  The kernel follows that: when launched with
+// programmatic stream serialization it draws the first shuffle while the preceding kernel
+// of the stream (the previous round's aggregation, which still reads the old table) runs,
+// and waits for it only before the first write to the table.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -41,6 +47,8 @@ k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __re
     extern __shared__ __align__(16) unsigned char sp_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int w = blockIdx.x * (blockDim.x >> 5) + warp;
+    // the next kernel of the stream may be scheduled as soon as SMs have room for it
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (w >= N) return;
     unsigned char* mine = sp_smem + (size_t)warp * per_worker_bytes;
     int32_t* perm = reinterpret_cast<int32_t*>(mine);
@@ -51,6 +59,7 @@ k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __re
     int M = N - 1;
     if (MASKED) {
         if (!online.get(w)) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             for (long long i = lane; i < (long long)S * R; i += 32) idx[(size_t)w * S * R + i] = -1;
             return;
         }
@@ -95,6 +104,8 @@ k_select_peers(uint64_t seed, uint32_t round, int N, int S, int R, int32_t* __re
             }
         }
         __syncwarp();
+        // first write to the table ahead: the preceding kernel must be done with the old one
+        if (e == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
         int pos = 0;
         while (pos < M && done < total) {
             int take = R - nc;
