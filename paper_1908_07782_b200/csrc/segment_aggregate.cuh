@@ -653,10 +653,17 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         // What the first tile needs is worked out, and the launch parameters it reads are
         // brought into the constant cache, before the wait: after it only the copy is left.
         const int l0_first = (int)((p.p_begin + (long long)blockIdx.x * p.T) / p.L);
-        asm volatile("" ::"l"(p.n_tiles), "l"(p.sched), "r"(p.stage_bytes), "r"(p.stage_off), "r"(l0_first));
-        wait_for_preceding_kernel();
         const uint32_t my_dst_off = (uint32_t)((a * p.nbx + b) * block_bytes + class_base * p.row_bytes);
         const int tile_cols_per_box = p.T / p.nbx;
+        // In a short kernel (fewer than 32 tiles per CTA) three quarters of the tiles are dealt
+        // out in fixed rounds (see below); the first ring always is.
+        long long static_rounds = stages;
+        if (p.n_tiles < 32LL * gridDim.x) static_rounds = (p.n_tiles * 3 / 4) / gridDim.x;
+        if (static_rounds < stages) static_rounds = stages;
+        const long long n_static = static_rounds * gridDim.x;
+        asm volatile("" ::"l"(p.n_tiles), "l"(p.sched), "l"(n_static), "r"(p.stage_bytes), "r"(p.stage_off),
+                     "r"(l0_first), "r"(my_dst_off), "r"(tile_cols_per_box));
+        wait_for_preceding_kernel();
         // Tiles are handed out dynamically: SMs differ by some 10 % in the HBM bandwidth they
         // get, and with a fixed share of tiles the slowest CTA would set the kernel time.  The
         // first ring of tiles is fixed (tile blockIdx.x + i * gridDim.x fills stage i), so that
@@ -668,14 +675,10 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         // for the atomic just sent into the other), hence the loop is unrolled by two.
         long long n = 0;
         long long tile = blockIdx.x;
-        // In a short kernel (fewer than 32 tiles per CTA) three quarters of the tiles are dealt
-        // out in fixed rounds as well: a claim is one more global operation in the producer's
-        // path, which is the critical one there.  (Measured: 1 % faster with 7 tiles per CTA,
-        // 1.3 % slower with hundreds, where the claims cost nothing and balance more.)
-        long long static_rounds = stages;
-        if (p.n_tiles < 32LL * gridDim.x) static_rounds = (p.n_tiles * 3 / 4) / gridDim.x;
-        if (static_rounds < stages) static_rounds = stages;
-        const long long n_static = static_rounds * gridDim.x;
+        // In a short kernel three quarters of the tiles are dealt out in fixed rounds as well: a
+        // claim is one more global operation in the producer's path, which is the critical one
+        // there.  (Measured: 1 % faster with 7 tiles per CTA, 1.3 % slower with hundreds, where
+        // the claims cost nothing and balance more.)
         bool open = true;                // false once a claim came back beyond the last tile
         // segment of the current tile's first column: a CTA's tiles come in ascending order,
         // so it is stepped forward instead of divided out per tile
@@ -949,6 +952,9 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                 if (++xb == p.nbx) { xb = 0; ++row; }
             }
         }
+        // The fused step rewrote the stage with ordinary stores; the copy that refills it goes
+        // through the asynchronous proxy, so the two are ordered by a proxy fence.
+        if (SGD) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
     }
