@@ -663,7 +663,10 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         const long long n_static = static_rounds * gridDim.x;
         asm volatile("" ::"l"(p.n_tiles), "l"(p.sched), "l"(n_static), "r"(p.stage_bytes), "r"(p.stage_off),
                      "r"(l0_first), "r"(my_dst_off), "r"(tile_cols_per_box));
-        wait_for_preceding_kernel();
+        // The wait for the preceding kernel comes as late as it can: the first step arms its
+        // barrier and writes its metadata (shared memory only) before it, so that after the
+        // wait nothing but the copy instruction itself is left to issue.
+        bool waited = false;
         // Tiles are handed out dynamically: SMs differ by some 10 % in the HBM bandwidth they
         // get, and with a fixed share of tiles the slowest CTA would set the kernel time.  The
         // first ring of tiles is fixed (tile blockIdx.x + i * gridDim.x fills stage i), so that
@@ -690,7 +693,9 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             const int s = (int)(n % stages);
             const uint32_t ph = (uint32_t)((n / stages) & 1);
             const bool last = tile >= p.n_tiles;
-            if (n + 2 >= static_rounds && open && !last && lane == 0) next2 = atomicAdd(&p.sched->next, 1ULL);
+            const bool claim = n + 2 >= static_rounds && open && !last;
+            if (claim && !waited) { wait_for_preceding_kernel(); waited = true; }   // global access ahead
+            if (claim && lane == 0) next2 = atomicAdd(&p.sched->next, 1ULL);
             if (!mbar_wait_patient(smem_u32(&hdr->empty[s]), ph ^ 1u)) { staged_fail(1); return false; }
             const long long t0 = tile * (long long)p.T;
             const uint32_t bar = smem_u32(&hdr->full[s]);
@@ -708,6 +713,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             __syncwarp();
             ++n;
             if (last) return false;
+            if (!waited) { wait_for_preceding_kernel(); waited = true; }
             if (issuer)
                 tma_load_2d(smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) + my_dst_off, my_map,
                             (int)(t0 + (long long)b * tile_cols_per_box), 0, bar);
@@ -728,6 +734,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             // register that step n - 1 was given as `next2`
             while (step(claim_a, claim_b) && step(claim_b, claim_a)) {}
         }
+        if (!waited) wait_for_preceding_kernel();
         // Leave last: every stage this warp armed must have landed before the CTA's
         // shared memory can be released, even if the consumers gave up.
         if (lane == 0) {
