@@ -40,8 +40,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="2", help="1..5 or a workload name (default: 2)")
     ap.add_argument("--impl", default="combo", choices=["combo", "reference"])
-    ap.add_argument("--op", default="round", choices=["round", "divergence"],
-                    help="round: the synchronization round (default); divergence: the Eq. 7 diagnostic alone")
+    ap.add_argument("--op", default="round", choices=["round", "divergence", "pull"],
+                    help="round: the synchronization round (default); divergence: the Eq. 7 diagnostic alone; "
+                         "pull: the worker-sharded round (workers spread over the ranks' GPUs, segments "
+                         "pulled from peer memory)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graphs", action="store_true", help="never replay short steps from CUDA graphs")
@@ -255,6 +257,81 @@ def run_divergence(args, wl):
     return 0
 
 
+# ------------------------------------------------------------------ worker-sharded round (extra line)
+def run_pull(args, wl):
+    """Times ShardedFederation.round: every rank hosts N/world workers in symmetric memory and
+    forms their new models with combo_segment_aggregate_rows, loading the pulled segments
+    from the owning GPU (Section 3).  With one rank every pull is a local load."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_1908_07782_b200 as combo
+    from paper_1908_07782_b200 import sharding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29531")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    e = elem_bytes(wl)
+    dtype = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    weights = synth.make_weights(wl, dev)
+    fed = sharding.ShardedFederation(wl.N, wl.P, wl.S, wl.R, dtype, weights=weights)
+    x = synth.make_params(wl, dev)                     # same seeds on every rank: take the hosted rows
+    fed.rows().copy_(x[fed.w_begin:fed.w_end])
+    del x
+    stream = torch.cuda.current_stream()
+    for t in range(max(args.warmup, 3)):
+        fed.round(wl.sampler_seed, t)
+    torch.cuda.synchronize()
+    dist.barrier()
+    a = torch.cuda.Event(enable_timing=True)
+    b = torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    steps = args.steps
+    for t in range(steps):
+        fed.round(wl.sampler_seed, 100 + t)
+    b.record(stream)
+    torch.cuda.synchronize()
+    dist.barrier()
+    ms = torch.tensor([a.elapsed_time(b) / steps], device=dev, dtype=torch.float64)
+    dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    ms = float(ms)
+    combo.combo_device_status()
+    if rank == 0:
+        idx_np = fed.idx.cpu().numpy()
+        traffic = sharding.pull_traffic(idx_np, world, wl.P, e)
+        link = int((traffic.sum(axis=1) - np.diag(traffic)).max())      # most any one rank pulls over NVLink
+        n_local_max = -(-wl.N // world)
+        alg = (wl.R + 2) * n_local_max * wl.P * e                        # per GPU: R+1 reads (no reuse), 1 write
+        peak, src = FALLBACK_HBM_GBS, "fallback"
+        mp = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(mp):
+            peak, src = float(json.load(open(mp))["hbm_gbs"]), "measured"
+        ach = alg / (ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "op": "worker_sharded_round", "value": wl.N * wl.P / (ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "strong", "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "N": wl.N, "P": wl.P, "S": wl.S, "R": wl.R,
+                       "workers_per_gpu": n_local_max, "parallelism": "workers sharded x%d" % world,
+                       "step": "barrier + peer selection + pull aggregation (1 round)"},
+            "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                         "traffic": None, "peak_source": src, "kernel": "k_pull_aggregate",
+                         "algorithmic_bytes_per_launch": alg,
+                         "nvlink_bytes_per_round_max_rank": link,
+                         "nvlink_gbs_max_rank": link / (ms * 1e-3) / 1e9},
+            "gpu_launches": 2 * steps,
+        }
+        print(json.dumps(line))
+    dist.destroy_process_group()
+    return 0
+
+
 # ------------------------------------------------------------------ our arm
 def main():
     args = parse_args()
@@ -268,6 +345,8 @@ def main():
         return run_reference(args, wl)
     if args.op == "divergence":
         return run_divergence(args, wl)
+    if args.op == "pull":
+        return run_pull(args, wl)
 
     import torch
     import torch.distributed as dist

@@ -140,6 +140,32 @@ combo_status combo_segment_aggregate_cols(const void* params_in, const void* gra
                                           void* stream);
 
 /*
+ * Worker-sharded form -- Section 3 "Segmented Pulling" (Eq. 2) followed by
+ * Eq. 3, for workers spread over several GPUs of one node.  d_rows: DEVICE
+ * array of N pointers, d_rows[j] = flat model of worker j (P elements, 16-byte
+ * aligned), in this GPU's memory or in a peer GPU's memory that is mapped
+ * into this process (peer access / symmetric memory).  The call forms the new
+ * models of the n_local workers w_begin .. w_begin + n_local - 1 that this
+ * GPU hosts and writes them to out, [n_local][out_pitch] (out_pitch >= P
+ * elements, out_pitch * elem_bytes a multiple of 16; must not overlap any
+ * row).  A pull is a plain load of W_k[l] from where worker k lives: per
+ * hosted worker exactly R segments per segment index cross to this GPU, as in
+ * the paper.  idx is the full [N][S][R] table (every GPU computes the same
+ * one from the seed), weights the full [N] array or NULL.  Same arithmetic and
+ * order as combo_segment_aggregate.  The caller orders the rounds: rows must
+ * be final before the call (Section 4.1: a worker sends after its local
+ * update) and must not be overwritten while any GPU still reads them.
+ */
+combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, int64_t out_pitch,
+                                          int elem_bytes, const float* weights, const int32_t* idx,
+                                          int N, int64_t P, int S, int R, int w_begin, int n_local,
+                                          void* stream);
+
+/* Debug helper for the call above: *dev_flag (device int32) becomes 0 when all
+ * N row pointers are non-null and 16-byte aligned, else 1 + the first bad row. */
+combo_status combo_check_rows(const void* const* d_rows, int N, void* stream, int32_t* dev_flag);
+
+/*
  * Dynamic workers -- Section 4.2.
  *
  * combo_select_peers_online: a worker that is offline is not pulled from (the
@@ -261,7 +287,7 @@ combo_status combo_aggregation_divergence_noalloc(const void* models, const void
 combo_status combo_device_status(void);
 
 /* Which aggregation kernel the last combo_segment_aggregate* call on this
- * thread launched: 0 none, 1 direct gather, 2 shared-memory staged. */
+ * thread launched: 0 none, 1 direct gather, 2 shared-memory staged, 3 row pull. */
 int combo_last_kernel_path(void);
 
 /* Forces a path for the following calls on this thread: 0 automatic (default),

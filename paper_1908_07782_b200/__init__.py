@@ -4,7 +4,8 @@ from .binding import (ComboError, combo_aggregation_divergence, combo_aggregatio
                       combo_divergence_scratch_bytes, PATH_AUTO, PATH_DIRECT, PATH_STAGED, combo_device_status,  # noqa: F401
                       combo_last_kernel_path, combo_round_host, combo_segment_aggregate,
                       combo_segment_aggregate_bf16, combo_segment_aggregate_cols,
-                      combo_segment_aggregate_members, combo_segment_aggregate_sgd, combo_select_peers,
+                      combo_segment_aggregate_members, combo_segment_aggregate_rows, combo_check_rows,
+                      combo_segment_aggregate_sgd, combo_select_peers,
                       combo_select_peers_online,
                       combo_select_peers_default_stream, combo_set_kernel_path, combo_set_launch_overlap,
                       combo_set_tuning,

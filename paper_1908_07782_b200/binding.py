@@ -47,6 +47,8 @@ def load():
         "combo_segment_aggregate_cols": [vp, vp, f32, vp, i32, vp, vp, i32, i64, i32, i32, i64, i64,
                                          i64, vp],
         "combo_validate_idx": [vp, i32, i32, i32, vp, vp],
+        "combo_segment_aggregate_rows": [vp, vp, i64, i32, vp, vp, i32, i64, i32, i32, i32, i32, vp],
+        "combo_check_rows": [vp, i32, vp, vp],
         "combo_select_peers_online": [u64, u32, i32, i32, i32, vp, vp, vp],
         "combo_segment_aggregate_members": [vp, vp, i32, vp, vp, vp, i32, i64, i32, i32, vp],
         "combo_round_host": [vp, vp, f32, vp, i32, vp, u64, u32, i32, i32, i64, i32, i32, vp, vp, vp,
@@ -142,6 +144,23 @@ def _host_bytes(flags, N):
         return None, None
     buf = (ctypes.c_uint8 * N)(*[1 if bool(f) else 0 for f in flags])
     return buf, ctypes.cast(buf, ctypes.c_void_p)
+
+
+def combo_segment_aggregate_rows(rows, out, out_pitch, elem_bytes, weights, idx, N, P, S, R, w_begin, n_local,
+                                 stream=None):
+    """Worker-sharded Eq. 3: ``rows`` is a device int64 tensor of N row addresses (local or
+    peer memory), ``out`` holds the n_local hosted workers' new models, [n_local][out_pitch]."""
+    _check(load().combo_segment_aggregate_rows(_ptr(rows), _ptr(out), out_pitch, elem_bytes, _ptr(weights),
+                                               _ptr(idx), N, P, S, R, w_begin, n_local, _stream(stream)),
+           "combo_segment_aggregate_rows")
+    return out
+
+
+def combo_check_rows(rows, N, stream=None) -> int:
+    """0 when all N row addresses are non-null and 16-byte aligned, else 1 + the first bad row."""
+    flag = torch.zeros(1, dtype=torch.int32, device=rows.device)
+    _check(load().combo_check_rows(_ptr(rows), N, _stream(stream), _ptr(flag)), "combo_check_rows")
+    return int(flag.item())
 
 
 def combo_select_peers_online(seed, rnd, N, S, R, online, idx_out, stream=None):

@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libcombo_b200.so")
 SOURCES = [os.path.join(CSRC, "combo_b200.cu")]
-DEPENDS = SOURCES + [os.path.join(CSRC, f) for f in ("segment_aggregate.cuh", "select_peers.cuh", "divergence.cuh")] + [
+DEPENDS = SOURCES + [os.path.join(CSRC, f) for f in ("segment_aggregate.cuh", "select_peers.cuh", "divergence.cuh", "pull_aggregate.cuh")] + [
     os.path.join(INCLUDE, "combo_b200.h")]
 
 

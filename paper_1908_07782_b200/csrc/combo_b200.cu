@@ -11,6 +11,7 @@
 #include "segment_aggregate.cuh"
 #include "divergence.cuh"
 #include "select_peers.cuh"
+#include "pull_aggregate.cuh"
 
 namespace {
 
@@ -629,6 +630,65 @@ combo_status combo_segment_aggregate_members(const void* params_in, void* params
                                              int N, int64_t P, int S, int R, void* stream) {
     return aggregate_cols(params_in, nullptr, 0.0f, params_out, elem_bytes, weights, idx, N, P, S, R, 0, P, P, stream,
                           h_newcomer);
+}
+
+combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, int64_t out_pitch, int elem_bytes,
+                                          const float* weights, const int32_t* idx, int N, int64_t P, int S, int R,
+                                          int w_begin, int n_local, void* stream) {
+    if (elem_bytes != 4 && elem_bytes != 2) return COMBO_ERR_INVALID_ARG;
+    if (N < 1 || N > COMBO_MAX_WORKERS || S < 1 || S > COMBO_MAX_SEGMENTS || R < 0 || R > N - 1 || P < 1)
+        return COMBO_ERR_INVALID_ARG;
+    if (w_begin < 0 || n_local < 1 || w_begin + n_local > N) return COMBO_ERR_INVALID_ARG;
+    if (!d_rows || !out || (R > 0 && !idx) || !aligned16(out)) return COMBO_ERR_INVALID_ARG;
+    if (out_pitch < P || (out_pitch * elem_bytes) % 16 != 0) return COMBO_ERR_INVALID_ARG;
+    DeviceInfo* dev = nullptr;
+    combo_status rc = device_info(&dev);
+    if (rc != COMBO_OK) return rc;
+    combo::PullParams p;
+    memset(&p, 0, sizeof(p));
+    p.rows = d_rows;
+    p.out = static_cast<unsigned char*>(out);
+    p.weights = weights;
+    p.idx = idx;
+    p.P = P;
+    p.L = (P + S - 1) / S;
+    p.out_pitch = out_pitch;
+    p.N = N; p.S = S; p.R = R;
+    p.w_begin = w_begin;
+    p.n_local = n_local;
+    const int V = 16 / elem_bytes;
+    const long long groups = (P + V - 1) / V;
+    // about eight resident CTAs per SM over all hosted workers together
+    long long bx = (groups + 255) / 256;
+    long long cap = ((long long)dev->sms * 8 + n_local - 1) / n_local;
+    if (cap < 1) cap = 1;
+    if (bx > cap) bx = cap;
+    const dim3 grid((unsigned)bx, (unsigned)n_local);
+    const size_t smem = (size_t)N * sizeof(void*);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaSuccess;
+    if (elem_bytes == 4) {
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(combo::k_pull_aggregate<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) combo::k_pull_aggregate<4><<<grid, 256, smem, st>>>(p);
+    } else {
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(combo::k_pull_aggregate<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) combo::k_pull_aggregate<2><<<grid, 256, smem, st>>>(p);
+    }
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "pull aggregation launch");
+    t_last_path = 3;
+    return COMBO_OK;
+}
+
+combo_status combo_check_rows(const void* const* d_rows, int N, void* stream, int32_t* dev_flag) {
+    if (!d_rows || N < 1 || !dev_flag) return COMBO_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(dev_flag, 0, sizeof(int32_t), st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    combo::k_check_rows<<<(N + 255) / 256, 256, 0, st>>>(d_rows, N, dev_flag);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "check_rows launch");
+    return COMBO_OK;
 }
 
 combo_status combo_validate_idx(const int32_t* idx, int N, int S, int R, void* stream, int32_t* dev_flag) {

@@ -1,0 +1,55 @@
+"""Host side of the worker-sharded round: who hosts whom, what crosses which link
+(Section 3: a worker pulls S*R segments, one model's worth per replica)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1908_07782_b200 import sharding
+
+
+@pytest.mark.parametrize("N,world", [(8, 1), (8, 2), (30, 4), (31, 4), (128, 8), (9, 8)])
+def test_worker_ranges_partition_the_workers(N, world):
+    seen = []
+    sizes = []
+    for r in range(world):
+        a, b = sharding.worker_range(r, world, N)
+        sizes.append(b - a)
+        seen += list(range(a, b))
+        for w in range(a, b):
+            assert sharding.owner_of(w, world, N) == r
+    assert seen == list(range(N))
+    assert max(sizes) - min(sizes) <= 1
+
+
+@pytest.mark.parametrize("P,S", [(40, 4), (25_557_032, 10), (7, 9), (23_520_842, 16)])
+def test_segment_lengths_follow_the_oracle_bounds(P, S):
+    lens = sharding.segment_lengths(P, S)
+    lo, hi = oracle.segment_bounds(P, S)
+    assert (lens == np.asarray(hi) - np.asarray(lo)).all()
+    assert lens.sum() == P
+
+
+def test_pull_traffic_counts_every_pulled_segment_once():
+    N, S, R, P, world, e = 32, 8, 3, 11_689_512, 4, 4
+    idx = oracle.select_peers(1, 0, N, S, R)
+    t = sharding.pull_traffic(idx, world, P, e)
+    # every worker pulls R whole models' worth of segments (Section 3, "Model Replica")
+    assert t.sum() == N * R * P * e
+    for a in range(world):
+        lo, hi = sharding.worker_range(a, world, N)
+        assert t[a].sum() == (hi - lo) * R * P * e
+    # brute force over the table for one pair of ranks
+    lens = sharding.segment_lengths(P, S) * e
+    want = 0
+    for w in range(*sharding.worker_range(1, world, N)):
+        for l in range(S):
+            for k in idx[w, l]:
+                if sharding.owner_of(int(k), world, N) == 3:
+                    want += lens[l]
+    assert t[1, 3] == want
+
+
+def test_one_rank_pulls_nothing_over_the_links():
+    idx = oracle.select_peers(1, 0, 8, 4, 2)
+    t = sharding.pull_traffic(idx, 1, 1_048_576, 4)
+    assert t.shape == (1, 1) and t[0, 0] == 8 * 2 * 1_048_576 * 4
