@@ -411,14 +411,20 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
         p.stage_off = p.mean_off + 2u * combo::kDivTile * 4u;
         p.m = m;
         const long long budget = (long long)dev->smem_optin - p.stage_off - 256;
-        // tile and box: the widest of which two stages fit; with row phases one box of 256
+        // tile: the widest whose stage stays within 64 KB (at least 64 columns if two stages
+        // fit at all); tiles beyond 256 columns are made of 256-column boxes.  With row phases
+        // one box of at most 256 columns.
         int TC = 0, box = 0;
         if (word) {
-            for (int c = combo::kDivTile; c >= 64; c >>= 1)
+            for (int c = combo::kDivBox; c >= 64; c >>= 1)
                 if (2LL * p.narr * N * c * EB <= budget) { TC = c - V; box = c; break; }
         } else {
-            for (int c = combo::kDivTile; c >= 64; c >>= 1)
-                if (2LL * p.narr * N * c * EB <= budget) { TC = box = c; break; }
+            for (int c = combo::kDivTile; c >= 64; c >>= 1) {
+                const long long stage = (long long)p.narr * N * c * EB;
+                if (2 * stage > budget || p.narr * (c > combo::kDivBox ? c / combo::kDivBox : 1) > 32) continue;
+                if (stage <= 64 * 1024 || c == 64 || c <= combo::kDivBox) { TC = c; break; }
+            }
+            box = TC > combo::kDivBox ? combo::kDivBox : TC;
         }
         combo::TileMaps maps;
         bool ok = TC > 0;
@@ -427,7 +433,7 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
                 ok = encode_class_map(&maps.map[a][j], a == 0 ? p.models : p.src, EB, j, m, N, P, P, box);
         if (ok) {
             p.row_bytes = box * EB;
-            p.stage_bytes = (unsigned)(p.narr * N * p.row_bytes);
+            p.stage_bytes = (unsigned)(p.narr * N * p.row_bytes) * (unsigned)(word ? 1 : TC / box);
             const int fit = (int)(budget / p.stage_bytes);
             // two tiles are in the consumers' hands at a time: three stages keep a load in flight
             int stages = (int)((112 * 1024) / p.stage_bytes);
@@ -447,6 +453,8 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
         if (e == cudaSuccess)                                                                                   \
             combo::k_divergence_staged<EBV, TCV, WV><<<nblocks, combo::kStagedThreads, smem, st>>>(p, maps);    \
     }
+            COMBO_DIV_LAUNCH(4, 1024, false) COMBO_DIV_LAUNCH(4, 512, false)
+            COMBO_DIV_LAUNCH(2, 1024, false) COMBO_DIV_LAUNCH(2, 512, false)
             COMBO_DIV_LAUNCH(4, 256, false) COMBO_DIV_LAUNCH(4, 128, false) COMBO_DIV_LAUNCH(4, 64, false)
             COMBO_DIV_LAUNCH(2, 256, false) COMBO_DIV_LAUNCH(2, 128, false) COMBO_DIV_LAUNCH(2, 64, false)
             COMBO_DIV_LAUNCH(4, 252, true) COMBO_DIV_LAUNCH(4, 124, true) COMBO_DIV_LAUNCH(4, 60, true)

@@ -19,7 +19,8 @@ namespace combo {
 
 constexpr int kDivSlots = 16;                          // rows a consumer warp can own
 constexpr int kDivMaxStagedN = kDivSlots * kConsumerWarps;
-constexpr int kDivTile = 256;                          // widest tile in columns = one TMA box
+constexpr int kDivBox = 256;                           // widest TMA box in columns
+constexpr int kDivTile = 1024;                         // widest tile in columns (four boxes)
 
 struct DivParams {
     const unsigned char* models;
@@ -31,8 +32,10 @@ struct DivParams {
     unsigned coef_off, rowoff_off, part_off, mean_off, stage_off, stage_bytes;
 };
 
-// TC = columns per tile.  Rows that are 16-byte aligned: 256, 128 or 64 (the widest of
-// which two stages fit), threads work on 128-bit vectors.  WORD: rows whose pitch is only a
+// TC = columns per tile.  Rows that are 16-byte aligned: 64 to 1024 (the widest whose stage
+// stays within 64 KB; tiles wider than 256 columns are staged as several boxes, which keeps
+// the per-tile costs -- a consumer-wide barrier, the producer's bookkeeping -- small against
+// the data when there are few rows), threads work on 128-bit vectors.  WORD: rows whose pitch is only a
 // multiple of 4 bytes are staged per row class with their phase (see the aggregation
 // kernel), TC = 256 - 16/e, and threads work on 4-byte words at the row's phase.
 template <int EB, int TC, bool WORD, bool PIPE = !WORD>
@@ -41,7 +44,10 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
     constexpr int UB = WORD ? 4 : 16;                  // bytes a thread takes at a time
     constexpr int EPU = UB / EB;                       // elements in them
     constexpr int NU = TC * EB / UB;                   // such units per row per tile
-    constexpr int NUP = NU <= 16 ? 16 : NU <= 32 ? 32 : NU <= 64 ? 64 : NU <= 128 ? 128 : 256;
+    constexpr int NBX = TC > kDivBox ? TC / kDivBox : 1;  // boxes per tile
+    constexpr int UPB = NU / NBX;                      // units per row held by one box
+    constexpr int NUP = NU <= 16 ? 16 : NU <= 32 ? 32 : NU <= 64 ? 64 : NU <= 128 ? 128 : NU <= 256 ? 256 : 512;
+    static_assert(NU <= kConsumerThreads, "a tile has more units than there are consumer threads");
     constexpr int G = kConsumerThreads / NUP;          // row groups of phase A
     constexpr int PSTR = NUP * EPU;                    // floats per row group in `part`
     extern __shared__ __align__(128) unsigned char smem[];
@@ -79,13 +85,16 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        const int a = lane / p.m, j = lane - a * p.m;
-        const bool issuer = lane < p.narr * p.m && j < N;
+        // lane -> one TMA box per tile: (array a, x-box b, class j)
+        const int per_arr = NBX * p.m;
+        const int a = lane / per_arr, rem = lane - a * per_arr;
+        const int b = rem / p.m, j = rem - b * p.m;
+        const bool issuer = lane < p.narr * per_arr && j < N;
         int class_base = 0;
         for (int q = 0; q < j; ++q) class_base += (N - q + p.m - 1) / p.m;
         const CUtensorMap* my_map = &maps.map[issuer ? a : 0][issuer ? j : 0];
         if (issuer) asm volatile("prefetch.tensormap [%0];" ::"l"(my_map) : "memory");
-        const uint32_t my_dst_off = (uint32_t)(a * block_bytes + class_base * p.row_bytes);
+        const uint32_t my_dst_off = (uint32_t)((a * NBX + b) * block_bytes + class_base * p.row_bytes);
         long long n = 0;
         for (long long tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % stages);
@@ -96,7 +105,7 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
             __syncwarp();
             if (issuer)
                 tma_load_2d(smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) + my_dst_off, my_map,
-                            (int)(tile * TC), 0, bar);
+                            (int)(tile * TC) + b * (TC / NBX), 0, bar);
         }
         if (lane == 0) {
             const long long first = n > stages ? n - stages : 0;
@@ -118,6 +127,8 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
 #pragma unroll
     for (int s = 0; s < kDivSlots; ++s) acc[s] = 0.0;
 
+    // byte offset of unit u of a row inside an array's part of a stage (its box, then its place)
+    auto unit_off = [&](int u) { return NBX == 1 ? u * UB : (u / UPB) * block_bytes + (u % UPB) * UB; };
     // one unit of a staged row as EPU binary32 values
     auto load_unit = [](const unsigned char* q, float (&x)[EPU]) {
         if constexpr (!WORD) {
@@ -170,7 +181,7 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
         if (i < n_my) {
             const int s = (int)(i % stages);
             if (!mbar_wait(smem_u32(&hdr->full[s]), (uint32_t)((i / stages) & 1))) { staged_fail(13); return; }
-            const unsigned char* xsrc = smem + p.stage_off + (size_t)s * p.stage_bytes + (p.narr - 1) * block_bytes;
+            const unsigned char* xsrc = smem + p.stage_off + (size_t)s * p.stage_bytes + (p.narr - 1) * NBX * block_bytes;
             float* pt = part + (i & 1) * (G * PSTR);
             // (A) weighted column sums of this thread's row group; columns past the end of the
             // rows were zero-filled by the TMA unit and contribute nothing anywhere below
@@ -180,7 +191,7 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
                 for (int e = 0; e < EPU; ++e) a[e] = 0.0f;
                 for (int j = ag; j < N; j += G) {
                     float x[EPU];
-                    load_unit(xsrc + rowoff[j] + au * UB, x);
+                    load_unit(xsrc + rowoff[j] + unit_off(au), x);
                     const float c = coef[j];
 #pragma unroll
                     for (int e = 0; e < EPU; ++e) a[e] = fmaf(c, x[e], a[e]);
@@ -189,12 +200,14 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
             }
         }
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(14); return; }
-        if (i < n_my && ctid < TC) {
+        if (i < n_my) {
             const float* pt = part + (i & 1) * (G * PSTR);
-            float m = 0.0f;
+            for (int c = ctid; c < TC; c += kConsumerThreads) {
+                float m = 0.0f;
 #pragma unroll
-            for (int g = 0; g < G; ++g) m = __fadd_rn(m, pt[g * PSTR + ctid]);
-            mean[(i & 1) * kDivTile + ctid] = m;
+                for (int g = 0; g < G; ++g) m = __fadd_rn(m, pt[g * PSTR + c]);
+                mean[(i & 1) * kDivTile + c] = m;
+            }
         }
         if (!PIPE) {
             // unpipelined form: the means of tile i must be complete before its deviations
@@ -215,7 +228,7 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
 #pragma unroll
                     for (int u = lane; u < NU; u += 32) {
                         float x[EPU], mu[EPU];
-                        load_unit(row + u * UB, x);
+                        load_unit(row + unit_off(u), x);
                         load_floats(mn + u * EPU, mu);
 #pragma unroll
                         for (int e = 0; e < EPU; ++e) {

@@ -54,6 +54,8 @@ CASES = [
     (64, 30_000, torch.float32),                  # two arrays of 64 rows: half-width tiles
     (200, 20_000, torch.float32),                 # too many rows for two staged tiles: fallback
     (300, 4_096, torch.bfloat16),                 # more than 256 workers
+    (16, 1_500_004, torch.float32),               # few rows: tiles of two boxes, several per CTA, ragged end
+    (4, 700_012, torch.bfloat16),                 # tiles of four boxes
 ]
 
 
