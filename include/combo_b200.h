@@ -9,6 +9,15 @@
  * device, calls only enqueue work on the given stream and never synchronise,
  * and the library allocates nothing.
  *
+ * Library-owned device memory: a 4-byte status word (combo_device_status) and
+ * a ring of 256 tile dispensers, 16 bytes each, of which every launch of the
+ * staged aggregation kernel takes the next one (its CTAs draw their tiles
+ * from it and the last one to leave clears it).  Launches that are in flight
+ * at the same time therefore hold different dispensers, as long as fewer
+ * than 256 launches separate them; a CUDA graph keeps the dispensers its
+ * kernels were captured with, so two DIFFERENT graphs captured a multiple of
+ * 256 launches apart must not run concurrently.
+ *
  * Notation follows the paper: n = N workers, S segments, R model replicas,
  * |D_j| dataset size of worker j, P_l the set of workers providing segment l.
  *
