@@ -834,6 +834,10 @@ combo_status combo_device_status(void) {
     if (v != 0) {
         int zero = 0;
         cudaMemcpyToSymbol(combo::g_dev_status, &zero, sizeof(int));
+        // a kernel that gave up may have left its tile dispenser half used: clear the ring
+        // (the device is idle here), so that the launch that next takes that slot starts clean
+        static const combo::TileSlot clean[combo::kTileSlots] = {};
+        cudaMemcpyToSymbol(combo::g_tile_slots, clean, sizeof(clean));
         snprintf(t_cuda_err, sizeof(t_cuda_err), "bounded wait gave up at site %d", v);
         return COMBO_ERR_DEVICE_TIMEOUT;
     }
