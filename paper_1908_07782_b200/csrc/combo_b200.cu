@@ -745,7 +745,7 @@ combo_status combo_round_host(const void* h_params_in, const void* h_grads, floa
     // through ALL rounds on its own.  Chunks are therefore pipelined over three streams:
     // chunk c+1 is copied in and chunk c-1 copied out while chunk c is aggregated.
     const size_t total = (size_t)N * pitch_bytes;
-    int K = (int)((total + (64u << 20) - 1) / (64u << 20));
+    int K = (int)((total + (8u << 20) - 1) / (8u << 20));     // chunks of at least 8 MB, at most kPipeChunks
     if (K > kPipeChunks) K = kPipeChunks;
     if (K < 1) K = 1;
     int64_t cw = ((P + K - 1) / K + 63) / 64 * 64;        // chunk width, 16-byte aligned starts
