@@ -514,7 +514,7 @@ combo_status noalloc_scratch(double** out) {
 }
 
 // Streams and events of the host-memory entry point, created on its first call on a device.
-constexpr int kPipeChunks = 16;
+constexpr int kPipeChunks = 32;
 struct HostPipe {
     bool ready;
     cudaStream_t s_in, s_out;
