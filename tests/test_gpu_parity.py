@@ -327,3 +327,19 @@ def test_round_from_host_memory_in_chunks(P, fused):
     combo.combo_round_host(hx, hg, 0.01, hout, 4, hw, 5, 0, 1, N, P, S, R, d_in, d_g, d_out, d_w, d_idx)
     check_against_oracle(hx[:, a:b].contiguous(), hout[:, a:b].contiguous(), idx0, S, R, weights=hw,
                          grads=hg[:, a:b].contiguous() if fused else None, lr=0.01, P=P, p_begin=a)
+
+
+def test_largest_worker_count():
+    # N at the library's limit (COMBO_MAX_WORKERS): sampler bit-exact, aggregation through the
+    # direct kernel (too many rows to stage), and one more worker is refused
+    N, P, S, R = 8192, 96, 2, 3
+    idx = gpu_select(7, 4, N, S, R)
+    idx_np = oracle.select_peers(7, 4, N, S, R)
+    assert (idx.cpu().numpy() == idx_np).all()
+    x, _, counts = _inputs(N, P, torch.float32, 5)
+    out, used = gpu_aggregate(x, idx, S, R, weights=counts)
+    assert used == combo.PATH_DIRECT
+    check_against_oracle(x, out, idx_np, S, R, weights=counts)
+    with pytest.raises(combo.ComboError) as e:
+        combo.combo_select_peers(7, 4, N + 1, S, R, torch.empty((N + 1, S, R), dtype=torch.int32, device=DEV))
+    assert e.value.status == 1
