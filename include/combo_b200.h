@@ -304,8 +304,8 @@ int combo_last_kernel_path(void);
 void combo_set_kernel_path(int path);
 
 /* Expert knob for the staged kernel, this thread only: tile width in elements
- * (a multiple of 256 up to 2048; rows whose byte pitch is
- * not a multiple of 16 always use 256 - 16/elem_bytes) and number of pipeline
+ * (a multiple of 256 up to 2048; for rows whose byte pitch is not a multiple
+ * of 16 every 256 asked for become 256 - 16/elem_bytes) and number of pipeline
  * stages; 0 = chosen automatically.  A tile that cannot be honoured makes
  * the call fall back to the direct kernel. */
 void combo_set_tuning(int tile_elems, int stages);

@@ -162,17 +162,21 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     // the coefficient table holds every segment when that is small (no rebuilds on the way,
     // which matters for short kernels), else two segments at a time
     const unsigned entry = (unsigned)combo::table_entry_bytes(rmax);
-    const int tab_slots = ((unsigned long long)p.S * p.N * entry <= 24u * 1024u && p.S >= 2) ? p.S : 2;
-    const unsigned table = round_up((unsigned)tab_slots * p.N * entry, 128);
+    int tab_slots = ((unsigned long long)p.S * p.N * entry <= 24u * 1024u && p.S >= 2) ? p.S : 2;
+    unsigned table = round_up((unsigned)tab_slots * p.N * entry, 128);
     const long long budget = (long long)dev.smem_optin - header - table - 256;
 
     // candidate tiles: (T, box_w, nbx)
     struct Cand { int T, box_w, nbx; };
-    Cand cands[combo::kMaxBoxes + 1];
+    Cand cands[combo::kMaxBoxes + 2];
     int nc = 0;
     if (unaligned) {
-        cands[nc++] = {256 - V, 256, 1};
+        // every box carries 256 - V columns of the tile plus room for the row phase
+        for (int n = 1; n <= combo::kMaxBoxes; ++n) cands[nc++] = {(256 - V) * n, 256, n};
     } else {
+        // with very many binary32 rows two stages of 256 columns do not fit: a half-width box
+        // (512 bytes per row, still a whole item per row) keeps such inputs on the staged path
+        if (EB == 4) cands[nc++] = {128, 128, 1};
         for (int n = 1; n <= combo::kMaxBoxes; ++n) cands[nc++] = {256 * n, 256, n};
     }
     auto stage_bytes = [&](const Cand& c) { return (long long)narr * c.nbx * p.N * c.box_w * EB; };
@@ -183,7 +187,7 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     int pick = -1;
     if (t_tile > 0) {
         for (int i = 0; i < nc; ++i)
-            if (cands[i].T == t_tile && feasible(cands[i])) pick = i;
+            if ((unaligned ? cands[i].nbx * 256 == t_tile : cands[i].T == t_tile) && feasible(cands[i])) pick = i;
         if (pick < 0) return plan;
     } else {
         // The widest tile whose stage stays within 64 KB and that still leaves every CTA some
@@ -211,6 +215,17 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     if (stages > combo::kMaxStages) stages = combo::kMaxStages;
     if (stages > fit) stages = fit;
     if (stages < 2) return plan;
+    // a larger table that still fits beside the stages chosen is taken whole as well (a rebuild
+    // costs two consumer barriers and a round trip to the peer table: it shows in kernels of
+    // a hundred microseconds with many segments)
+    if (tab_slots < p.S) {
+        const unsigned long long whole = round_up((unsigned)((unsigned long long)p.S * p.N * entry), 128);
+        if ((unsigned long long)p.S * p.N * entry < (1u << 20) &&
+            (long long)(whole - table) <= budget - (long long)stages * stage_bytes(c)) {
+            tab_slots = p.S;
+            table = (unsigned)whole;
+        }
+    }
     p.T = c.T;
     p.m = m;
     p.nbx = c.nbx;

@@ -761,7 +761,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     uint32_t csync_phase = 0;
     int cached_l0 = -1;
     // A unit of consumer work is one row of one x-box: CPB chunks of 512 bytes.
-    constexpr int CPB = (EB == 4) ? 2 : 1;         // boxes are 256 elements wide
+    constexpr int CPB = (EB == 4) ? 2 : 1;         // boxes are at most 256 elements wide
     const int box_payload = (p.T / p.nbx) * EB;    // tile bytes per row held by one x-box
     const int n_units = N * p.nbx;
     const int upw = (n_units + kConsumerWarps - 1) / kConsumerWarps;
@@ -872,24 +872,48 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
 
         int row = row_begin, xb = xb_begin;
         if (GB < 16 && interior) {
-            // word mode: the tile is one box, a unit is a whole row of it, and only the last
-            // piece of a row can lie outside the payload (a loop-invariant lane predicate)
+            // word mode: a unit is a whole row of a box, and only the last piece of it can lie
+            // outside the box's payload (a loop-invariant lane predicate)
             if constexpr (GB < 16) {
                 RowCtx<RMAX> c;
-                const unsigned char* ent = tab0 + (size_t)u_begin * ENT;
-                unsigned char* orow = p.out + (size_t)u_begin * pitch_bytes + (size_t)t0 * EB + lane * GB;
                 const uint32_t lane_base = stage_s + lane * GB;
                 const bool last_on = (CPB - 1) * 512 + lane * GB + (PIECES - 1) * PSTRIDE < box_payload;
+                if (p.nbx == 1) {
+                    // the tile is one box (many rows): a unit is a row
+                    const unsigned char* ent = tab0 + (size_t)u_begin * ENT;
+                    unsigned char* orow = p.out + (size_t)u_begin * pitch_bytes + (size_t)t0 * EB + lane * GB;
 #pragma unroll 2
-                for (int u = u_begin; u < u_end; ++u) {
-                    load_entry<RMAX>(ent, c);
+                    for (int u = u_begin; u < u_end; ++u) {
+                        load_entry<RMAX>(ent, c);
 #pragma unroll
-                    for (int ch = 0; ch < CPB - 1; ++ch)
-                        item_box<EB, GB, RMAX, (RT >= 0), false>(lane_base + ch * 512, c, R, orow + ch * 512, true);
-                    item_box<EB, GB, RMAX, (RT >= 0), true>(lane_base + (CPB - 1) * 512, c, R,
-                                                            orow + (CPB - 1) * 512, last_on);
-                    ent += ENT;
-                    orow += pitch_bytes;
+                        for (int ch = 0; ch < CPB - 1; ++ch)
+                            item_box<EB, GB, RMAX, (RT >= 0), false>(lane_base + ch * 512, c, R, orow + ch * 512, true);
+                        item_box<EB, GB, RMAX, (RT >= 0), true>(lane_base + (CPB - 1) * 512, c, R,
+                                                                orow + (CPB - 1) * 512, last_on);
+                        ent += ENT;
+                        orow += pitch_bytes;
+                    }
+                } else {
+                    // several boxes per tile (few rows): rows outside, boxes inside
+                    const int nbx = p.nbx;
+                    const unsigned char* ent = tab0 + (size_t)row * ENT;
+                    unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
+                    int u = u_begin;
+                    while (u < u_end) {
+                        load_entry<RMAX>(ent, c);
+                        for (; xb < nbx && u < u_end; ++xb, ++u) {
+                            const uint32_t ubase = lane_base + xb * block_bytes;
+                            unsigned char* uout = orow + xb * box_payload;
+#pragma unroll
+                            for (int ch = 0; ch < CPB - 1; ++ch)
+                                item_box<EB, GB, RMAX, (RT >= 0), false>(ubase + ch * 512, c, R, uout + ch * 512, true);
+                            item_box<EB, GB, RMAX, (RT >= 0), true>(ubase + (CPB - 1) * 512, c, R,
+                                                                    uout + (CPB - 1) * 512, last_on);
+                        }
+                        xb = 0;
+                        ent += ENT;
+                        orow += pitch_bytes;
+                    }
                 }
             }
         } else if (interior) {
@@ -907,7 +931,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                     unsigned char* uout = orow + xb * box_payload;
 #pragma unroll
                     for (int ch = 0; ch < CPB; ++ch)
-                        if (GB == 16 || ch * 512 < box_payload)
+                        if (ch * 512 < box_payload)
                             item_fast<EB, GB, RMAX, (RT >= 0)>(ubase + ch * 512, c, R, uout + ch * 512, pmask[ch]);
                 }
                 xb = 0;
@@ -920,6 +944,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             for (int u = u_begin; u < u_end; ++u) {
 #pragma unroll 1
                 for (int ch = 0; ch < CPB; ++ch) {
+                    if (ch * 512 >= box_payload) continue;               // half-width boxes hold one item per row
                     const int ib = xb * box_payload + ch * 512;          // byte offset of the item in the row
                     const uint32_t ubase = stage_s + xb * block_bytes + ch * 512 + lane * GB;
                     bool done = false;

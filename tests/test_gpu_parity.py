@@ -183,6 +183,11 @@ def test_staged_unaligned_rows(P, dtype):
     (6, 70_000, 7, 5, torch.bfloat16),      # R without a specialised kernel
     (200, 3_000, 4, 3, torch.float32),      # many workers, short rows (segments shorter than a tile)
     (130, 40_000, 2, 2, torch.bfloat16),    # more than 128 workers
+    (150, 30_000, 4, 3, torch.float32),     # so many binary32 rows that only half-width boxes fit two stages
+    (176, 20_004, 3, 4, torch.float32),
+    (24, 300_002, 5, 4, torch.bfloat16),    # few rows with differing phases: word-mode tiles of several boxes
+    (6, 400_001, 4, 2, torch.float32),      # the same for binary32 (4 row classes)
+    (10, 200_003, 3, 3, torch.bfloat16),    # odd bf16 pitch (8 classes, 2-byte granule), several boxes
 ])
 def test_staged_odd_shapes(N, P, S, R, dtype):
     x, grads, counts = _inputs(N, P, dtype, 77)
