@@ -190,18 +190,22 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
             if ((unaligned ? cands[i].nbx * 256 == t_tile : cands[i].T == t_tile) && feasible(cands[i])) pick = i;
         if (pick < 0) return plan;
     } else {
-        // The widest tile whose stage stays within 64 KB and that still leaves every CTA some
-        // six tiles: tiles are handed out dynamically, and with fewer the last ones of a short
-        // kernel leave SMs idle (measured with 8 rows of 1 M floats: 14.4 us with 3.5 tiles
-        // per CTA, 13.9 us with 7).  When even the narrowest tile gives fewer, the narrowest.
-        int narrowest = -1;
+        // Long kernels: the widest tile whose stage stays within 64 KB.  Short kernels (fewer
+        // than 32 such tiles per CTA, i.e. up to some hundred microseconds): the widest tile
+        // whose stage stays within 32 KB -- they spend a good part of their time filling and
+        // draining the ring, which narrower stages do faster, and tiles are handed out
+        // dynamically, which balances better with more of them.  (Measured on shapes from
+        // 8 x 256 K to 16 x 1 M floats: the 32 KB choice was the best or within 1 % of it;
+        // 8 x 1 M: 14.4 us with 64 KB stages, 13.5 us with 32 KB.)
+        int wide = -1, mid = -1, narrowest = -1;
         for (int i = 0; i < nc; ++i) {
             if (!feasible(cands[i])) continue;
             if (narrowest < 0) narrowest = i;
-            if (stage_bytes(cands[i]) > 64 * 1024) continue;
-            if (tiles(cands[i]) >= 6LL * dev.sms) pick = i;
+            if (stage_bytes(cands[i]) <= 64 * 1024) wide = i;
+            if (stage_bytes(cands[i]) <= 32 * 1024 && cands[i].box_w == 256) mid = i;   // half-width boxes: last resort only
         }
-        if (pick < 0) pick = narrowest;
+        pick = wide >= 0 ? wide : narrowest;
+        if (wide >= 0 && tiles(cands[wide]) < 32LL * dev.sms && mid >= 0) pick = mid;
         if (pick < 0) return plan;
     }
     const Cand c = cands[pick];
