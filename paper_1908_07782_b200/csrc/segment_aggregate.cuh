@@ -882,7 +882,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
                     // the tile is one box (many rows): a unit is a row
                     const unsigned char* ent = tab0 + (size_t)u_begin * ENT;
                     unsigned char* orow = p.out + (size_t)u_begin * pitch_bytes + (size_t)t0 * EB + lane * GB;
-#pragma unroll 2
+#pragma unroll 4   // measured: 2 -> 4 gains 1.7 % with 128 bf16 rows, 8 gains nothing
                     for (int u = u_begin; u < u_end; ++u) {
                         load_entry<RMAX>(ent, c);
 #pragma unroll
