@@ -379,6 +379,11 @@ def main():
     sets = [[x0, torch.empty_like(x0)]]
     for _ in range(nsets - 1):
         sets.append([x0.clone(), torch.empty_like(x0)])
+    if args.warm and pair_bytes < 512e6:
+        # the same pair eight times over, so that a replayed graph holds as many launches as
+        # in the rotating case (a graph of one short kernel would time the graph launch)
+        nsets = 8
+        sets = sets * 8
     bufs = sets[0]
     weights = synth.make_weights(wl, dev)
     grads = synth.make_grads(wl, 0, dev, seed=1000 + seed) if wl.fused_sgd else None
@@ -591,7 +596,7 @@ def main():
                        "l2": ("inputs larger than L2 (%.2f GB in + out per round)" % (pair_bytes / 1e9)
                               if pair_bytes >= 512e6 else
                               "WARM: one buffer pair of %.0f MB, served from L2 where it fits" % (pair_bytes / 1e6))
-                       if nsets == 1 else "rotating over %d buffer pairs (%.0f MB) so that each step reads HBM"
+                       if (nsets == 1 or args.warm) else "rotating over %d buffer pairs (%.0f MB) so that each step reads HBM"
                        % (nsets, nsets * pair_bytes / 1e6),
                        "kernel_path": {1: "direct", 2: "staged"}.get(kernel_path, "?"),
                        "launch": "CUDA graph replay (step shorter than its CPU launch cost)" if use_graphs
