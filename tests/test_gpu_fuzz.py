@@ -37,3 +37,35 @@ def test_random_shapes(seed):
         check_against_oracle(x[:, c0:c1].contiguous(), a[:, c0:c1].contiguous(), idx_np, S, R, weights=w,
                              grads=grads[:, c0:c1].contiguous() if fused else None, lr=0.01, P=P, p_begin=c0)
     combo.combo_device_status()
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_long_rows(seed):
+    # few rows, long vectors: tens of tiles per CTA, so that most tiles come from the
+    # dispenser, with every alignment residue and segment boundaries inside tiles
+    rng = np.random.default_rng(5000 + seed)
+    dtype = torch.float32 if rng.random() < 0.6 else torch.bfloat16
+    N = int(rng.choice([2, 4, 5, 8, 12, 16, 24]))
+    R = int(rng.integers(1, min(N - 1, 6) + 1))
+    S = int(rng.choice([1, 3, 4, 7, 10, 32]))
+    P = int(rng.integers(1_000_000, 3_000_000)) + int(rng.integers(0, 16))
+    fused = dtype == torch.float32 and rng.random() < 0.4
+    weighted = rng.random() < 0.5
+    g = torch.Generator().manual_seed(seed)
+    x = (torch.randn(N, P, generator=g) * 0.05).to(dtype).to(DEV)
+    grads = (torch.randn(N, P, generator=g) * 1e-3).to(DEV) if fused else None
+    w = torch.randint(500, 1501, (N,), generator=g).float().to(DEV) if weighted else None
+    idx_np = oracle.select_peers(seed, 3, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    a, used = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_STAGED)
+    assert used == combo.PATH_STAGED, (N, P, S, R, dtype, fused)
+    b, _ = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_DIRECT)
+    assert torch.equal(a, b), (N, P, S, R, dtype, fused)
+    L = -(-P // S)
+    windows = [(0, 2000), (max(P - 2000, 0), P)]
+    if S > 1:
+        windows.append((L - 1000, min(L + 1000, P)))        # across the first segment boundary
+    for (c0, c1) in windows:
+        check_against_oracle(x[:, c0:c1].contiguous(), a[:, c0:c1].contiguous(), idx_np, S, R, weights=w,
+                             grads=grads[:, c0:c1].contiguous() if fused else None, lr=0.01, P=P, p_begin=c0)
+    combo.combo_device_status()
