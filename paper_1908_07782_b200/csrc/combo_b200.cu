@@ -309,16 +309,18 @@ cudaError_t launch_staged(const AggParams& p, const combo::TileMaps& maps, const
 
 cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo& dev, cudaStream_t st) {
     const int V = 16 / EB;
-    const long long items = ((p.width + V - 1) / V + 1) * (long long)p.N;
-    long long blocks = (items + 255) / 256;
-    const long long cap = (long long)dev.sms * 32;
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
+    const long long groups = (p.width + V - 1) / V + 1;
+    // x over the groups of a row, y = worker; about 32 resident CTAs per SM over all workers
+    long long bx = (groups + 255) / 256;
+    long long cap = ((long long)dev.sms * 32 + p.N - 1) / p.N;
+    if (cap < 1) cap = 1;
+    if (bx > cap) bx = cap;
+    const dim3 grid((unsigned)bx, (unsigned)p.N);
     if (EB == 4) {
-        if (sgd) combo::k_direct<4, true><<<(int)blocks, 256, 0, st>>>(p);
-        else combo::k_direct<4, false><<<(int)blocks, 256, 0, st>>>(p);
+        if (sgd) combo::k_direct<4, true><<<grid, 256, 0, st>>>(p);
+        else combo::k_direct<4, false><<<grid, 256, 0, st>>>(p);
     } else {
-        combo::k_direct<2, false><<<(int)blocks, 256, 0, st>>>(p);
+        combo::k_direct<2, false><<<grid, 256, 0, st>>>(p);
     }
     return cudaGetLastError();
 }

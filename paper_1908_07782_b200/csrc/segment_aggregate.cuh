@@ -351,12 +351,11 @@ template <int EB, bool SGD>
 __global__ void __launch_bounds__(256) k_direct(const AggParams p) {
     constexpr int V = ElemOps<EB>::V;
     const long long G = (p.width + V - 1) / V + 1;      // groups per row, phase spill included
-    const long long items = G * (long long)p.N;
     const bool rows_aligned = (p.pitch % V) == 0;
-    for (long long it = blockIdx.x * 256LL + threadIdx.x; it < items; it += (long long)gridDim.x * 256LL) {
-        const int w = (int)(it / G);
-        const long long g = it - (long long)w * G;
-        const int a_w = (int)(((long long)w * p.pitch) & (V - 1));
+    // grid: x strides over the groups of a row, y = worker
+    const int w = blockIdx.y;
+    const int a_w = (int)(((long long)w * p.pitch) & (V - 1));
+    for (long long g = blockIdx.x * 256LL + threadIdx.x; g < G; g += (long long)gridDim.x * 256LL) {
         const long long c0 = g * V - a_w;
         const long long lo = c0 < 0 ? 0 : c0;
         const long long hi = (c0 + V > p.width) ? p.width : c0 + V;
