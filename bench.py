@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--P", type=int, default=0, help="override the vector length (scaled-down runs)")
     ap.add_argument("--N", type=int, default=0, help="override the number of workers")
     ap.add_argument("--rounds", type=int, default=0, help="override the rounds per step")
+    ap.add_argument("--S", type=int, default=0, help="override the number of segments")
+    ap.add_argument("--R", type=int, default=-1, help="override the number of replicas (peers per segment)")
     ap.add_argument("--tile", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--warm", action="store_true",
@@ -340,10 +342,12 @@ def main():
     args = parse_args()
     from paper_1908_07782_b200 import synth
     wl = synth.get_workload(args.workload)
-    if args.P or args.N or args.rounds:
+    if args.P or args.N or args.rounds or args.S or args.R >= 0:
         import dataclasses
         wl = dataclasses.replace(wl, P=args.P or wl.P, N=args.N or wl.N, rounds=args.rounds or wl.rounds,
-                                 name="%s@N=%d,P=%d" % (wl.name, args.N or wl.N, args.P or wl.P))
+                                 S=args.S or wl.S, R=args.R if args.R >= 0 else wl.R,
+                                 name="%s@N=%d,P=%d,S=%d,R=%d" % (wl.name, args.N or wl.N, args.P or wl.P,
+                                                                 args.S or wl.S, args.R if args.R >= 0 else wl.R))
     if args.impl == "reference":
         return run_reference(args, wl)
     if args.op == "divergence":

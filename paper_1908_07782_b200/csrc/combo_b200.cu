@@ -157,7 +157,8 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     plan.gb = !unaligned ? 16 : (EB == 4 ? 4 : ((p.pitch % 2 == 0) ? 4 : 2));
     // the kernel is specialised on R for 1..4 except on the rarely used granules
     plan.rt = (p.R >= 1 && p.R <= 4 && (plan.gb == 16 || (EB == 2 && plan.gb == 4))) ? p.R : -1;
-    const int rmax = plan.rt >= 0 ? plan.rt : combo::kStagedMaxR;
+    if (p.R > combo::kGenericR) plan.rt = -2;                       // the wide unspecialised kernel
+    const int rmax = plan.rt >= 0 ? plan.rt : (plan.rt == -2 ? combo::kStagedMaxR : combo::kGenericR);
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
     // the coefficient table holds every segment when that is small (no rebuilds on the way,
     // which matters for short kernels), else two segments at a time
@@ -284,6 +285,7 @@ cudaError_t launch_staged_r(const AggParams& p, const combo::TileMaps& maps, con
         case 2: return launch_staged_inst<EB, GB, SGD, 2>(p, maps, plan, st);
         case 3: return launch_staged_inst<EB, GB, SGD, 3>(p, maps, plan, st);
         case 4: return launch_staged_inst<EB, GB, SGD, 4>(p, maps, plan, st);
+        case -2: return launch_staged_inst<EB, GB, SGD, -2>(p, maps, plan, st);
         default: return launch_staged_inst<EB, GB, SGD, -1>(p, maps, plan, st);
     }
 }
@@ -291,6 +293,7 @@ cudaError_t launch_staged_r(const AggParams& p, const combo::TileMaps& maps, con
 template <int EB, int GB, bool SGD>
 cudaError_t launch_staged_generic(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan,
                                   cudaStream_t st) {
+    if (plan.rt == -2) return launch_staged_inst<EB, GB, SGD, -2>(p, maps, plan, st);
     return launch_staged_inst<EB, GB, SGD, -1>(p, maps, plan, st);
 }
 

@@ -43,7 +43,8 @@ constexpr int kConsumerWarps = COMBO_CONSUMER_WARPS;
 constexpr int kConsumerThreads = 32 * kConsumerWarps;
 constexpr int kStagedThreads = 32 + kConsumerThreads;
 constexpr int kMaxStages = 8;
-constexpr int kStagedMaxR = 8;
+constexpr int kStagedMaxR = 16;            // most replicas the staged kernel takes (Section 5.2 sweeps R up to 16)
+constexpr int kGenericR = 8;               // replicas of the unspecialised kernel; beyond: the wide one
 constexpr int kMaxClasses = 8;
 constexpr int kMaxBoxes = 8;              // x-boxes per tile
 constexpr uint32_t kWaitCap = 1u << 23;   // polls before a wait is declared dead
@@ -604,7 +605,9 @@ template <int EB, int GB, bool SGD, int RT>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     constexpr int V = ElemOps<EB>::V;
-    constexpr int RMAX = (RT >= 0) ? RT : kStagedMaxR;
+    // RT: the number of replicas the kernel is specialised on, -1 = any up to kGenericR,
+    // -2 = any up to kStagedMaxR
+    constexpr int RMAX = (RT >= 0) ? RT : (RT == -2 ? kStagedMaxR : kGenericR);
     constexpr int ENT = table_entry_bytes(RMAX);
     constexpr int PIECES = 16 / GB;            // pieces a lane owns per item
     constexpr int PSTRIDE = 32 * GB;           // bytes between a lane's pieces

@@ -16,7 +16,7 @@ def test_random_shapes(seed):
     rng = np.random.default_rng(1000 + seed)
     dtype = torch.float32 if rng.random() < 0.6 else torch.bfloat16
     N = int(rng.choice([2, 3, 5, 8, 13, 16, 31, 32, 48, 64, 96, 128, 160]))
-    R = int(rng.integers(0, min(N - 1, 9) + 1))
+    R = int(rng.integers(0, min(N - 1, 17) + 1))
     S = int(rng.choice([1, 2, 3, 4, 7, 8, 10, 16, 32]))
     P = int(rng.integers(20_000, 400_000 // max(N // 16, 1)))
     P += int(rng.integers(0, 16))                       # every alignment residue

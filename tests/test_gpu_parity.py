@@ -101,8 +101,11 @@ MEDIUM = [
     (64, 9_992, 10, 4, torch.float32, False),     # last segment shorter
     (16, 33_000, 32, 4, torch.float32, False),
     (5, 50_000, 3, 4, torch.float32, True),       # R = N-1
-    (12, 30_000, 5, 8, torch.float32, True),      # largest R the staged kernel takes
-    (12, 30_000, 5, 9, torch.float32, True),      # beyond it: direct kernel
+    (12, 30_000, 5, 8, torch.float32, True),      # largest R of the narrow unspecialised kernel
+    (12, 30_000, 5, 9, torch.float32, True),      # the wide one
+    (20, 30_000, 10, 16, torch.float32, True),    # largest R the staged kernel takes (Section 5.2 sweeps R to 16)
+    (20, 30_002, 10, 16, torch.bfloat16, False),  # the same with differing row phases
+    (20, 30_000, 3, 17, torch.float32, True),     # beyond it: direct kernel
     (7, 30_000, 3, 0, torch.float32, False),      # R = 0
     (1, 30_000, 3, 0, torch.float32, False),      # a single worker
     (128, 5_002, 16, 4, torch.bfloat16, False),   # row pitch = 4 mod 16 bytes (granule 4)
@@ -121,7 +124,7 @@ def test_aggregate_medium_both_kernels(N, P, S, R, dtype, weighted, path):
     idx_np = oracle.select_peers(1, 2, N, S, R)
     idx = torch.from_numpy(idx_np).to(DEV) if R > 0 else None
     out, used = gpu_aggregate(x, idx, S, R, weights=weights, path=path)
-    if path == combo.PATH_STAGED and R <= 8:
+    if path == combo.PATH_STAGED and R <= 16:
         assert used == combo.PATH_STAGED
     check_against_oracle(x, out, idx_np, S, R, weights=weights)
     if R == 0:
