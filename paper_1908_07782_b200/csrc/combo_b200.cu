@@ -155,8 +155,9 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     if ((unsigned long long)m * (unsigned long long)pitch_bytes >= (1ull << 40)) return plan;
     if ((unsigned long long)p.width + V >= (1ull << 32)) return plan;
     plan.gb = !unaligned ? 16 : (EB == 4 ? 4 : ((p.pitch % 2 == 0) ? 4 : 2));
-    // the kernel is specialised on R for 1..4 except on the rarely used granules
-    plan.rt = (p.R >= 1 && p.R <= 4 && (plan.gb == 16 || (EB == 2 && plan.gb == 4))) ? p.R : -1;
+    // the kernel is specialised on R for 1..4 and 8 (the values Section 5.2 sweeps, with 16)
+    // except on the rarely used granules
+    plan.rt = (((p.R >= 1 && p.R <= 4) || p.R == 8) && (plan.gb == 16 || (EB == 2 && plan.gb == 4))) ? p.R : -1;
     if (p.R > combo::kGenericR) plan.rt = -2;                       // the wide unspecialised kernel
     const int rmax = plan.rt >= 0 ? plan.rt : (plan.rt == -2 ? combo::kStagedMaxR : combo::kGenericR);
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
@@ -285,6 +286,7 @@ cudaError_t launch_staged_r(const AggParams& p, const combo::TileMaps& maps, con
         case 2: return launch_staged_inst<EB, GB, SGD, 2>(p, maps, plan, st);
         case 3: return launch_staged_inst<EB, GB, SGD, 3>(p, maps, plan, st);
         case 4: return launch_staged_inst<EB, GB, SGD, 4>(p, maps, plan, st);
+        case 8: return launch_staged_inst<EB, GB, SGD, 8>(p, maps, plan, st);
         case -2: return launch_staged_inst<EB, GB, SGD, -2>(p, maps, plan, st);
         default: return launch_staged_inst<EB, GB, SGD, -1>(p, maps, plan, st);
     }
