@@ -296,11 +296,15 @@ combo_status combo_aggregation_divergence_noalloc(const void* models, const void
 combo_status combo_device_status(void);
 
 /* Which aggregation kernel the last combo_segment_aggregate* call on this
- * thread launched: 0 none, 1 direct gather, 2 shared-memory staged, 3 row pull. */
+ * thread launched: 0 none, 1 direct gather, 2 shared-memory staged (persistent
+ * CTAs, a ring of tiles), 3 row pull, 5 shared-memory staged with one tile per
+ * CTA (short inputs). */
 int combo_last_kernel_path(void);
 
 /* Forces a path for the following calls on this thread: 0 automatic (default),
- * 1 direct gather, 2 staged (falls back to direct where staging cannot apply). */
+ * 1 direct gather, 2 staged with persistent CTAs (falls back to direct where
+ * staging cannot apply), 5 staged with one tile per CTA (falls back to 2 where
+ * rows differ in their 16-byte phase or a tile does not fit). */
 void combo_set_kernel_path(int path);
 
 /* Expert knob for the staged kernel, this thread only: tile width in elements

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libcombo_b200.so")
 _lib = None
 
 COMBO_OK = 0
-PATH_AUTO, PATH_DIRECT, PATH_STAGED = 0, 1, 2
+PATH_AUTO, PATH_DIRECT, PATH_STAGED, PATH_TILE = 0, 1, 2, 5
 
 
 class ComboError(RuntimeError):

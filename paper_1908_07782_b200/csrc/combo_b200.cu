@@ -23,11 +23,13 @@ thread_local int t_force_path = 0;
 thread_local int t_tile = 0;
 thread_local int t_stages = 0;
 thread_local int t_overlap = 1;
+constexpr long long kTileMaxCtas = 1LL << 18;   // largest grid the one-tile-per-CTA kernel is chosen for
 
 struct DeviceInfo {
     int known;       // 0 unknown, 1 supported, -1 unsupported
     int sms;
     int smem_optin;
+    int smem_per_sm;
 };
 DeviceInfo g_dev[64];
 
@@ -43,13 +45,15 @@ combo_status device_info(DeviceInfo** out) {
     if (dev < 0 || dev >= 64) return COMBO_ERR_UNSUPPORTED;
     DeviceInfo& d = g_dev[dev];
     if (d.known == 0) {
-        int major = 0, sms = 0, smem = 0;
+        int major = 0, sms = 0, smem = 0, smem_sm = 0;
         if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess ||
             (e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
-            (e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+            (e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess)
             return cuda_fail(e, "cudaDeviceGetAttribute");
         d.sms = sms;
         d.smem_optin = smem;
+        d.smem_per_sm = smem_sm;
         d.known = (major == 10) ? 1 : -1;
     }
     if (d.known < 0) return COMBO_ERR_UNSUPPORTED;
@@ -153,7 +157,7 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     const bool unaligned = m > 1;
     if ((p.N + m - 1) / m > 256) return plan;                       // box rows
     if ((unsigned long long)m * (unsigned long long)pitch_bytes >= (1ull << 40)) return plan;
-    if ((unsigned long long)p.width + V >= (1ull << 32)) return plan;
+    if ((unsigned long long)p.width + 256 >= (1ull << 31)) return plan;   // TMA coordinates are signed 32-bit
     plan.gb = !unaligned ? 16 : (EB == 4 ? 4 : ((p.pitch % 2 == 0) ? 4 : 2));
     // the kernel is specialised on R for 1..4 and 8 (the values Section 5.2 sweeps, with 16)
     // except on the rarely used granules
@@ -312,6 +316,116 @@ cudaError_t launch_staged(const AggParams& p, const combo::TileMaps& maps, const
     return launch_staged_generic<2, 2, false>(p, maps, plan, st);
 }
 
+// Plan of the one-tile-per-CTA kernel (k_tile): rows that share one 16-byte phase only, one
+// stage, a table of two segments.  `short_enough` tells whether the automatic choice should
+// take it (few rows: small tiles, many CTAs per SM).
+StagedPlan plan_tile(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, const DeviceInfo& dev,
+                     bool* short_enough) {
+    StagedPlan plan = {false, 16, -1, 0, 0};
+    *short_enough = false;
+    const int V = 16 / EB;
+    const int narr = sgd ? 2 : 1;
+    if (p.R > combo::kStagedMaxR) return plan;
+    if ((p.pitch * EB) % 16 != 0) return plan;                      // one row class only
+    if (p.N > 256) return plan;                                     // box rows
+    if ((unsigned long long)p.pitch * EB >= (1ull << 40)) return plan;
+    if ((unsigned long long)p.width + 256 >= (1ull << 31)) return plan;   // TMA coordinates are signed 32-bit
+    plan.rt = ((p.R >= 1 && p.R <= 4) || p.R == 8) ? p.R : -1;
+    if (p.R > combo::kGenericR) plan.rt = -2;
+    const int rmax = plan.rt >= 0 ? plan.rt : (plan.rt == -2 ? combo::kStagedMaxR : combo::kGenericR);
+    const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
+    const unsigned table = round_up(2u * p.N * (unsigned)combo::table_entry_bytes(rmax), 128);
+    // Tile: at least 1 KB of every row (256 binary32 or 512 bfloat16 columns; shorter row
+    // pieces cost HBM efficiency) and at least 8 KB in all, else as small as possible: the
+    // smaller the tile, the more CTAs share an SM and the finer the hand-over between
+    // consecutive launches (measured on 2 to 32 rows of 1 M to 4 M elements: 8 rows of 1 M
+    // floats take 12.7 us with 8 KB tiles, 13.3 with 16 KB, 14.6 with 32 KB; tiles of 4 KB
+    // and less are far slower).  t_tile overrides.
+    int nbx = 0;
+    for (int n = 1; n <= combo::kMaxBoxes; ++n) {
+        if (256LL * n > p.L || narr * n > 32) break;
+        if (t_tile > 0) {
+            if (256 * n == t_tile) nbx = n;
+            continue;
+        }
+        nbx = n;
+        if (256 * n * EB >= 1024 && (long long)narr * n * p.N * 256 * EB >= 8 * 1024) break;
+    }
+    if (nbx == 0) return plan;
+    const long long stage = (long long)narr * nbx * p.N * 256 * EB;
+    const size_t smem = (size_t)header + table + (size_t)stage + 16;
+    if ((long long)smem > dev.smem_optin) return plan;
+    p.T = 256 * nbx;
+    p.m = 1;
+    p.nbx = nbx;
+    p.box_w = 256;
+    p.stages = 1;
+    p.row_bytes = 256 * EB;
+    p.stage_bytes = (unsigned)stage;
+    p.tab_off = header;
+    p.tab_slots = 2;
+    p.stage_off = header + table;
+    p.n_tiles = (p.width + p.T - 1) / p.T;
+    if (p.n_tiles > 0x7fffffffLL) return plan;
+    for (int a = 0; a < narr; ++a)
+        if (!encode_class_map(&maps.map[a][0], a == 0 ? p.in : p.grads, EB, 0, 1, p.N, p.pitch, p.width, 256))
+            return plan;
+    plan.smem = smem;
+    plan.grid = (int)p.n_tiles;
+    plan.ok = plan.grid > 0;
+    (void)V;
+    // Taken automatically where it measured faster than the persistent kernel's ring: tiles of
+    // 8 to 16 KB (up to 16 rows), which let a dozen or more CTAs share an SM, and at most two
+    // replicas.  (8 x 1 M floats, R = 2: 12.8 us against 13.6; 16 x 1 M: 23.2 against 24.4;
+    // 2 x 4 M, R = 1: 12.1 against 18.9.  With R = 3 or 4 the ring wins by 10 to 15 %, with 24
+    // and more rows it is as good or better, bfloat16 tiles of 8 KB lose 5 %.)
+    *short_enough = stage >= 8 * 1024 && stage <= 16 * 1024 && p.R <= 2 && (EB == 4 || stage == 16 * 1024) &&
+                    p.n_tiles <= kTileMaxCtas;
+    return plan;
+}
+
+template <int EB, bool SGD, int RT>
+cudaError_t launch_tile_inst(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan,
+                             cudaStream_t st) {
+    auto kern = combo::k_tile<EB, 16, SGD, RT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)plan.grid);
+    cfg.blockDim = dim3((unsigned)combo::kTileThreads);
+    cfg.dynamicSmemBytes = plan.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = t_overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, p, maps);
+}
+
+template <int EB, bool SGD>
+cudaError_t launch_tile_r(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan,
+                          cudaStream_t st) {
+    switch (plan.rt) {
+        case 1: return launch_tile_inst<EB, SGD, 1>(p, maps, plan, st);
+        case 2: return launch_tile_inst<EB, SGD, 2>(p, maps, plan, st);
+        case 3: return launch_tile_inst<EB, SGD, 3>(p, maps, plan, st);
+        case 4: return launch_tile_inst<EB, SGD, 4>(p, maps, plan, st);
+        case 8: return launch_tile_inst<EB, SGD, 8>(p, maps, plan, st);
+        case -2: return launch_tile_inst<EB, SGD, -2>(p, maps, plan, st);
+        default: return launch_tile_inst<EB, SGD, -1>(p, maps, plan, st);
+    }
+}
+
+cudaError_t launch_tile(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan, int EB, bool sgd,
+                        cudaStream_t st) {
+    if (EB == 4) return sgd ? launch_tile_r<4, true>(p, maps, plan, st) : launch_tile_r<4, false>(p, maps, plan, st);
+    return launch_tile_r<2, false>(p, maps, plan, st);
+}
+
 cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo& dev, cudaStream_t st) {
     const int V = 16 / EB;
     const long long groups = (p.width + V - 1) / V + 1;
@@ -330,6 +444,10 @@ cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo
     return cudaGetLastError();
 }
 
+// widest column range one launch takes: a multiple of 64 elements (shards start on 16-byte
+// boundaries) that keeps every TMA coordinate, box width included, below 2^31
+constexpr long long kMaxShardColumns = 1LL << 30;
+
 combo_status aggregate_cols(const void* in, const void* grads, float lr, void* out, int EB,
                             const float* weights, const int32_t* idx, int N, long long P_total, int S, int R,
                             long long p_begin, long long width, long long pitch, void* stream,
@@ -345,6 +463,20 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
     if ((unsigned long long)pitch > (1ull << 40) / (unsigned)N) return COMBO_ERR_INVALID_ARG;
     const size_t extent = (size_t)(((long long)(N - 1) * pitch + width) * EB);
     if (overlaps(in, out, extent) || (grads && overlaps(grads, out, extent))) return COMBO_ERR_ALIAS;
+
+    // The staged kernels address columns with signed 32-bit TMA coordinates.  Wider inputs are
+    // cut into column shards, which Eq. 3 allows (workers are coupled only at equal column).
+    if (width > kMaxShardColumns) {
+        for (long long c0 = 0; c0 < width; c0 += kMaxShardColumns) {
+            const long long w = width - c0 < kMaxShardColumns ? width - c0 : kMaxShardColumns;
+            combo_status rcs = aggregate_cols(static_cast<const char*>(in) + c0 * EB,
+                                              grads ? static_cast<const char*>(grads) + c0 * EB : nullptr, lr,
+                                              static_cast<char*>(out) + c0 * EB, EB, weights, idx, N, P_total, S, R,
+                                              p_begin + c0, w, pitch, stream, h_newcomer);
+            if (rcs != COMBO_OK) return rcs;
+        }
+        return COMBO_OK;
+    }
 
     DeviceInfo* dev = nullptr;
     combo_status rc = device_info(&dev);
@@ -371,6 +503,19 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
 
     bool want_staged = t_force_path != 1;
     if (t_force_path == 0 && (long long)N * width < (1 << 16)) want_staged = false;   // too small to pipeline
+    if (want_staged && t_force_path != 2) {
+        // short inputs: one tile per CTA, several CTAs per SM
+        combo::TileMaps maps;
+        AggParams q = p;
+        bool short_enough = false;
+        StagedPlan plan = plan_tile(q, maps, EB, sgd, *dev, &short_enough);
+        if (plan.ok && (short_enough || t_force_path == 5)) {
+            cudaError_t e = launch_tile(q, maps, plan, EB, sgd, st);
+            if (e != cudaSuccess) return cuda_fail(e, "tile aggregation launch");
+            t_last_path = 5;
+            return COMBO_OK;
+        }
+    }
     if (want_staged) {
         combo::TileMaps maps;
         StagedPlan plan = plan_staged(p, maps, EB, sgd, *dev);
@@ -872,7 +1017,7 @@ combo_status combo_device_status(void) {
 
 int combo_last_kernel_path(void) { return t_last_path; }
 
-void combo_set_kernel_path(int path) { t_force_path = (path == 1 || path == 2) ? path : 0; }
+void combo_set_kernel_path(int path) { t_force_path = (path == 1 || path == 2 || path == 5) ? path : 0; }
 
 void combo_set_tuning(int tile_elems, int stages) {
     t_tile = tile_elems > 0 ? tile_elems : 0;

@@ -486,6 +486,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// The same box brought into L2 only (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y)
+                 : "memory");
+}
+
 // 16 bytes, written and read as one vector (the producer's shared-memory operations queue
 // behind the consumers' stores, so each one saved shortens its per-tile path)
 struct alignas(16) TileMeta {
@@ -601,17 +607,242 @@ __device__ __forceinline__ void item_box(uint32_t base, const RowCtx<RMAX>& c, i
     PairStoreBox<EB, GB>::template run<LAST>(outp, acc, last_on);
 }
 
+// Fused local step on a staged tile, in place: x <- fma(-lr, g, x) for every staged row; the
+// gradients of the tile lie `bytes` behind the parameters.  Thread t of nthreads.
+__device__ __forceinline__ void sgd_step_in_place(unsigned char* stage, int bytes, float lr, int t, int nthreads) {
+    const int nvec = bytes / 16;
+    float4* xs = reinterpret_cast<float4*>(stage);
+    const float4* gs = reinterpret_cast<const float4*>(stage + (size_t)bytes);
+    const float nlr = -lr;
+    for (int v = t; v < nvec; v += nthreads) {
+        float4 x = xs[v];
+        const float4 g = gs[v];
+        x.x = fmaf(nlr, g.x, x.x); x.y = fmaf(nlr, g.y, x.y);
+        x.z = fmaf(nlr, g.z, x.z); x.w = fmaf(nlr, g.w, x.w);
+        xs[v] = x;
+    }
+}
+
+// Coefficient / offset table of `nslots` consecutive segments starting at l0_build, built by
+// `nthreads` threads of which the caller is number t: entry [slot][w] of ENT bytes.
+template <int EB, int RMAX>
+__device__ __forceinline__ void build_coef_table(const AggParams& p, unsigned char* tab, int R, int l0_build,
+                                                 int nslots, int t, int nthreads) {
+    constexpr int ENT = table_entry_bytes(RMAX);
+    const int N = p.N;
+    for (int q = t; q < nslots * N; q += nthreads) {
+        const int slot = q / N, w = q - slot * N;
+        const int l = l0_build + slot;
+        if (l < p.S) {
+            const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
+            float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
+            int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
+            // providers in the fixed order: the worker itself (unless it is a newcomer), then
+            // the peers ascending; a negative entry is a pull that found no online peer
+            int prov[RMAX + 1];
+            int np = 0;
+            if (!p.newcomer.get(w)) prov[np++] = w;
+            for (int r = 0; r < R; ++r) {
+                const int k = peers[r];
+                if (k >= 0) prov[np++] = k;
+            }
+            if (np == 0) prov[np++] = w;                 // nothing to aggregate: keep the own values
+            float den = p.weights ? p.weights[prov[0]] : 1.0f;
+            for (int i = 1; i < np; ++i) den = __fadd_rn(den, p.weights ? p.weights[prov[i]] : 1.0f);
+            for (int r = 0; r < np; ++r) {
+                const int k = prov[r];
+                cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                // staged row of worker k: classes are stored one after another
+                const int jk = k % p.m;
+                int base = 0;
+                for (int q2 = 0; q2 < jk; ++q2) base += (N - q2 + p.m - 1) / p.m;
+                const int phase = (int)(((long long)k * p.pitch * EB) & 15);
+                po[r] = (base + k / p.m) * p.row_bytes + phase;
+            }
+            // unused slots: coefficient zero on a row that is known to hold finite values
+            for (int r = np; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
+        }
+    }
+}
+
+// The share of a tile that one of `nwarps` warps works on.  A unit of work is one row of one
+// x-box: CPB chunks of 512 bytes; a warp takes a contiguous range of units.
+template <int EB, int GB>
+struct WarpShare {
+    static constexpr int CPB = (EB == 4) ? 2 : 1;         // boxes are at most 256 elements wide
+    static constexpr int PIECES = 16 / GB;                // pieces a lane owns per item
+    static constexpr int PSTRIDE = 32 * GB;               // bytes between a lane's pieces
+    int u_begin, u_end, row_begin, xb_begin;
+    int box_payload;                                      // tile bytes per row held by one x-box
+    size_t pitch_bytes;
+    unsigned pmask[CPB];    // store masks of the unit's chunks: bit i = piece i of this lane lies inside the payload
+    __device__ __forceinline__ WarpShare(const AggParams& p, int cw, int nwarps, int lane) {
+        box_payload = (p.T / p.nbx) * EB;
+        const int n_units = p.N * p.nbx;
+        const int upw = (n_units + nwarps - 1) / nwarps;
+        u_begin = cw * upw;
+        u_end = (cw + 1) * upw < n_units ? (cw + 1) * upw : n_units;
+        row_begin = u_begin / p.nbx;
+        xb_begin = u_begin - row_begin * p.nbx;
+        pitch_bytes = (size_t)p.pitch * EB;
+#pragma unroll
+        for (int ch = 0; ch < CPB; ++ch) {
+            pmask[ch] = 0;
+#pragma unroll
+            for (int i = 0; i < PIECES; ++i)
+                if (ch * 512 + lane * GB + i * PSTRIDE < box_payload) pmask[ch] |= 1u << i;
+        }
+    }
+};
+
+// One warp's share of a staged tile: Eq. 3 in the fixed order for every unit of `ws`, results
+// stored to the output rows.  `stage` holds the tile (its shared-window address is stage_s),
+// tab0 the table entries of segment l0 (those of l0 + 1 follow them), m_bnd is the local
+// column where segment l0 + 1 starts.
+template <int EB, int GB, int RT>
+__device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpShare<EB, GB>& ws,
+                                               const unsigned char* stage, uint32_t stage_s,
+                                               const unsigned char* tab0, long long tile, long long m_bnd,
+                                               int lane) {
+    constexpr int V = ElemOps<EB>::V;
+    constexpr int RMAX = (RT >= 0) ? RT : (RT == -2 ? kStagedMaxR : kGenericR);
+    constexpr int ENT = table_entry_bytes(RMAX);
+    constexpr int CPB = WarpShare<EB, GB>::CPB;
+    constexpr int PIECES = WarpShare<EB, GB>::PIECES;
+    constexpr int PSTRIDE = WarpShare<EB, GB>::PSTRIDE;
+    constexpr int EPP = GB / EB;               // elements per piece
+    const int N = p.N, R = (RT >= 0) ? RT : p.R;
+    const int block_bytes = N * p.row_bytes;               // one x-box of all rows
+    const int box_payload = ws.box_payload;
+    const size_t pitch_bytes = ws.pitch_bytes;
+    const int u_begin = ws.u_begin, u_end = ws.u_end;
+    const long long t0 = tile * (long long)p.T;
+    const long long t1 = (t0 + p.T < p.width) ? t0 + p.T : p.width;
+    const bool interior = (m_bnd >= t1) && (t0 + p.T <= p.width);   // one segment, whole tile
+
+    int row = ws.row_begin, xb = ws.xb_begin;
+    if (GB < 16 && interior) {
+        // word mode: a unit is a whole row of a box, and only the last piece of it can lie
+        // outside the box's payload (a loop-invariant lane predicate)
+        if constexpr (GB < 16) {
+            RowCtx<RMAX> c;
+            const uint32_t lane_base = stage_s + lane * GB;
+            const bool last_on = (CPB - 1) * 512 + lane * GB + (PIECES - 1) * PSTRIDE < box_payload;
+            if (p.nbx == 1) {
+                // the tile is one box (many rows): a unit is a row
+                const unsigned char* ent = tab0 + (size_t)u_begin * ENT;
+                unsigned char* orow = p.out + (size_t)u_begin * pitch_bytes + (size_t)t0 * EB + lane * GB;
+#pragma unroll 4   // measured: 2 -> 4 gains 1.7 % with 128 bf16 rows, 8 gains nothing
+                for (int u = u_begin; u < u_end; ++u) {
+                    load_entry<RMAX>(ent, c);
+#pragma unroll
+                    for (int ch = 0; ch < CPB - 1; ++ch)
+                        item_box<EB, GB, RMAX, (RT >= 0), false>(lane_base + ch * 512, c, R, orow + ch * 512, true);
+                    item_box<EB, GB, RMAX, (RT >= 0), true>(lane_base + (CPB - 1) * 512, c, R,
+                                                            orow + (CPB - 1) * 512, last_on);
+                    ent += ENT;
+                    orow += pitch_bytes;
+                }
+            } else {
+                // several boxes per tile (few rows): rows outside, boxes inside
+                const int nbx = p.nbx;
+                const unsigned char* ent = tab0 + (size_t)row * ENT;
+                unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
+                int u = u_begin;
+                while (u < u_end) {
+                    load_entry<RMAX>(ent, c);
+                    for (; xb < nbx && u < u_end; ++xb, ++u) {
+                        const uint32_t ubase = lane_base + xb * block_bytes;
+                        unsigned char* uout = orow + xb * box_payload;
+#pragma unroll
+                        for (int ch = 0; ch < CPB - 1; ++ch)
+                            item_box<EB, GB, RMAX, (RT >= 0), false>(ubase + ch * 512, c, R, uout + ch * 512, true);
+                        item_box<EB, GB, RMAX, (RT >= 0), true>(ubase + (CPB - 1) * 512, c, R,
+                                                                uout + (CPB - 1) * 512, last_on);
+                    }
+                    xb = 0;
+                    ent += ENT;
+                    orow += pitch_bytes;
+                }
+            }
+        }
+    } else if (interior) {
+        // every unit is whole and lies in segment l0: the lean loop, rows outside, boxes inside
+        RowCtx<RMAX> c;
+        const int nbx = p.nbx;
+        const unsigned char* ent = tab0 + (size_t)row * ENT;
+        unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
+        const uint32_t lane_base = stage_s + lane * GB;
+        int u = u_begin;
+        while (u < u_end) {
+            load_entry<RMAX>(ent, c);
+            for (; xb < nbx && u < u_end; ++xb, ++u) {
+                const uint32_t ubase = lane_base + xb * block_bytes;
+                unsigned char* uout = orow + xb * box_payload;
+#pragma unroll
+                for (int ch = 0; ch < CPB; ++ch)
+                    if (ch * 512 < box_payload)
+                        item_fast<EB, GB, RMAX, (RT >= 0)>(ubase + ch * 512, c, R, uout + ch * 512, ws.pmask[ch]);
+            }
+            xb = 0;
+            ent += ENT;
+            orow += pitch_bytes;
+        }
+    } else {
+        // last tile of the rows, or a tile holding a segment boundary: element by element,
+        // except whole 128-bit groups that lie in one segment
+        for (int u = u_begin; u < u_end; ++u) {
+#pragma unroll 1
+            for (int ch = 0; ch < CPB; ++ch) {
+                if (ch * 512 >= box_payload) continue;               // half-width boxes hold one item per row
+                const int ib = xb * box_payload + ch * 512;          // byte offset of the item in the row
+                const uint32_t ubase = stage_s + xb * block_bytes + ch * 512 + lane * GB;
+                bool done = false;
+                if (GB == 16) {
+                    const long long c0 = t0 + (ib + lane * 16) / EB;
+                    const bool whole = c0 + V <= p.width;
+                    const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
+                    if (whole && one_seg) {
+                        RowCtx<RMAX> cc;
+                        load_entry<RMAX>(tab0 + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
+                        item_fast<EB, GB, RMAX, (RT >= 0)>(
+                            ubase, cc, R, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
+                        done = true;
+                    }
+                }
+                if (!done) {
+#pragma unroll 1
+                    for (int i = 0; i < PIECES; ++i) {
+                        const int pin = ch * 512 + lane * GB + i * PSTRIDE;  // byte offset inside the box payload
+                        if (pin >= box_payload) continue;
+#pragma unroll 1
+                        for (int e = 0; e < EPP; ++e) {
+                            const long long col = t0 + (xb * box_payload + pin) / EB + e;
+                            if (col >= p.width) continue;
+                            const unsigned char* ent = tab0 + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
+                            const float* cf = reinterpret_cast<const float*>(ent);       // pairs
+                            const int* po = reinterpret_cast<const int*>(cf + 2 * (RMAX + 1));
+                            const unsigned char* eb = stage + xb * block_bytes + pin + e * EB;
+                            float acc = __fmul_rn(cf[0], ElemOps<EB>::load(eb + po[0]));
+                            for (int r = 1; r <= R; ++r)
+                                acc = fmaf(cf[2 * r], ElemOps<EB>::load(eb + po[r]), acc);
+                            ElemOps<EB>::store(p.out + (size_t)row * pitch_bytes + (size_t)col * EB, acc);
+                        }
+                    }
+                }
+            }
+            if (++xb == p.nbx) { xb = 0; ++row; }
+        }
+    }
+}
+
 template <int EB, int GB, bool SGD, int RT>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
-    constexpr int V = ElemOps<EB>::V;
     // RT: the number of replicas the kernel is specialised on, -1 = any up to kGenericR,
     // -2 = any up to kStagedMaxR
     constexpr int RMAX = (RT >= 0) ? RT : (RT == -2 ? kStagedMaxR : kGenericR);
     constexpr int ENT = table_entry_bytes(RMAX);
-    constexpr int PIECES = 16 / GB;            // pieces a lane owns per item
-    constexpr int PSTRIDE = 32 * GB;           // bytes between a lane's pieces
-    constexpr int EPP = GB / EB;               // elements per piece
     extern __shared__ __align__(128) unsigned char smem[];
     StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -762,70 +993,17 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     const int ctid = tid - 32;
     uint32_t csync_phase = 0;
     int cached_l0 = -1;
-    // A unit of consumer work is one row of one x-box: CPB chunks of 512 bytes.
-    constexpr int CPB = (EB == 4) ? 2 : 1;         // boxes are at most 256 elements wide
-    const int box_payload = (p.T / p.nbx) * EB;    // tile bytes per row held by one x-box
-    const int n_units = N * p.nbx;
-    const int upw = (n_units + kConsumerWarps - 1) / kConsumerWarps;
-    const int u_begin = cw * upw;
-    const int u_end = (cw + 1) * upw < n_units ? (cw + 1) * upw : n_units;
-    const int row_begin = u_begin / p.nbx, xb_begin = u_begin - row_begin * p.nbx;
+    const WarpShare<EB, GB> ws(p, cw, kConsumerWarps, lane);
     const uint32_t csync = smem_u32(&hdr->csync);
-    const size_t pitch_bytes = (size_t)p.pitch * EB;
-    // store masks of the unit's chunks: bit i = piece i of this lane lies inside the payload
-    unsigned pmask[CPB];
-#pragma unroll
-    for (int ch = 0; ch < CPB; ++ch) {
-        pmask[ch] = 0;
-#pragma unroll
-        for (int i = 0; i < PIECES; ++i)
-            if (ch * 512 + lane * GB + i * PSTRIDE < box_payload) pmask[ch] |= 1u << i;
-    }
 
-    // Coefficient / offset table of segments l0 and l0+1, built by all consumer threads.
-    auto build_table = [&](int l0_build, int nslots) {
-        for (int q = ctid; q < nslots * N; q += kConsumerThreads) {
-            const int slot = q / N, w = q - slot * N;
-            const int l = l0_build + slot;
-            if (l < p.S) {
-                const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
-                float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
-                int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
-                // providers in the fixed order: the worker itself (unless it is a newcomer), then
-                // the peers ascending; a negative entry is a pull that found no online peer
-                int prov[RMAX + 1];
-                int np = 0;
-                if (!p.newcomer.get(w)) prov[np++] = w;
-                for (int r = 0; r < R; ++r) {
-                    const int k = peers[r];
-                    if (k >= 0) prov[np++] = k;
-                }
-                if (np == 0) prov[np++] = w;                 // nothing to aggregate: keep the own values
-                float den = p.weights ? p.weights[prov[0]] : 1.0f;
-                for (int t = 1; t < np; ++t) den = __fadd_rn(den, p.weights ? p.weights[prov[t]] : 1.0f);
-                for (int r = 0; r < np; ++r) {
-                    const int k = prov[r];
-                    cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
-                    // staged row of worker k: classes are stored one after another
-                    const int jk = k % p.m;
-                    int base = 0;
-                    for (int q2 = 0; q2 < jk; ++q2) base += (N - q2 + p.m - 1) / p.m;
-                    const int phase = (int)(((long long)k * p.pitch * EB) & 15);
-                    po[r] = (base + k / p.m) * p.row_bytes + phase;
-                }
-                // unused slots: coefficient zero on a row that is known to hold finite values
-                for (int r = np; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
-            }
-        }
-    };
     // The first tile's table does not depend on the staged data: build it while the
     // first TMA loads are in flight.
     if ((long long)blockIdx.x < p.n_tiles) {
         if (whole_table) {
-            build_table(0, p.S);
+            build_coef_table<EB, RMAX>(p, tab, R, 0, p.S, ctid, kConsumerThreads);
         } else {
             cached_l0 = (int)((p.p_begin + (long long)blockIdx.x * p.T) / p.L);
-            build_table(cached_l0, 2);
+            build_coef_table<EB, RMAX>(p, tab, R, cached_l0, 2, ctid, kConsumerThreads);
         }
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(7); return; }
     }
@@ -847,151 +1025,99 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         if (!whole_table && m_l0 != cached_l0) {
             // table for segments l0 and l0+1 (rebuilt at most S times per CTA)
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(4); return; }
-            build_table(m_l0, 2);
+            build_coef_table<EB, RMAX>(p, tab, R, m_l0, 2, ctid, kConsumerThreads);
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
             cached_l0 = m_l0;
         }
 
         if (SGD) {
             // local step on the staged tile, in place: x <- fma(-lr, g, x), every row
-            const int nvec = p.nbx * block_bytes / 16;
-            float4* xs = reinterpret_cast<float4*>(stage);
-            const float4* gs = reinterpret_cast<const float4*>(stage + (size_t)p.nbx * block_bytes);
-            const float nlr = -p.lr;
-            for (int v = ctid; v < nvec; v += kConsumerThreads) {
-                float4 x = xs[v];
-                const float4 g = gs[v];
-                x.x = fmaf(nlr, g.x, x.x); x.y = fmaf(nlr, g.y, x.y);
-                x.z = fmaf(nlr, g.z, x.z); x.w = fmaf(nlr, g.w, x.w);
-                xs[v] = x;
-            }
+            sgd_step_in_place(stage, p.nbx * block_bytes, p.lr, ctid, kConsumerThreads);
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(6); return; }
         }
 
-        const long long t0 = tile * (long long)p.T;
-        const long long t1 = (t0 + p.T < p.width) ? t0 + p.T : p.width;
-        const bool interior = (m_bnd >= t1) && (t0 + p.T <= p.width);   // one segment, whole tile
+        aggregate_tile<EB, GB, RT>(p, ws, stage, stage_s, tab0, tile, m_bnd, lane);
 
-        int row = row_begin, xb = xb_begin;
-        if (GB < 16 && interior) {
-            // word mode: a unit is a whole row of a box, and only the last piece of it can lie
-            // outside the box's payload (a loop-invariant lane predicate)
-            if constexpr (GB < 16) {
-                RowCtx<RMAX> c;
-                const uint32_t lane_base = stage_s + lane * GB;
-                const bool last_on = (CPB - 1) * 512 + lane * GB + (PIECES - 1) * PSTRIDE < box_payload;
-                if (p.nbx == 1) {
-                    // the tile is one box (many rows): a unit is a row
-                    const unsigned char* ent = tab0 + (size_t)u_begin * ENT;
-                    unsigned char* orow = p.out + (size_t)u_begin * pitch_bytes + (size_t)t0 * EB + lane * GB;
-#pragma unroll 4   // measured: 2 -> 4 gains 1.7 % with 128 bf16 rows, 8 gains nothing
-                    for (int u = u_begin; u < u_end; ++u) {
-                        load_entry<RMAX>(ent, c);
-#pragma unroll
-                        for (int ch = 0; ch < CPB - 1; ++ch)
-                            item_box<EB, GB, RMAX, (RT >= 0), false>(lane_base + ch * 512, c, R, orow + ch * 512, true);
-                        item_box<EB, GB, RMAX, (RT >= 0), true>(lane_base + (CPB - 1) * 512, c, R,
-                                                                orow + (CPB - 1) * 512, last_on);
-                        ent += ENT;
-                        orow += pitch_bytes;
-                    }
-                } else {
-                    // several boxes per tile (few rows): rows outside, boxes inside
-                    const int nbx = p.nbx;
-                    const unsigned char* ent = tab0 + (size_t)row * ENT;
-                    unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
-                    int u = u_begin;
-                    while (u < u_end) {
-                        load_entry<RMAX>(ent, c);
-                        for (; xb < nbx && u < u_end; ++xb, ++u) {
-                            const uint32_t ubase = lane_base + xb * block_bytes;
-                            unsigned char* uout = orow + xb * box_payload;
-#pragma unroll
-                            for (int ch = 0; ch < CPB - 1; ++ch)
-                                item_box<EB, GB, RMAX, (RT >= 0), false>(ubase + ch * 512, c, R, uout + ch * 512, true);
-                            item_box<EB, GB, RMAX, (RT >= 0), true>(ubase + (CPB - 1) * 512, c, R,
-                                                                    uout + (CPB - 1) * 512, last_on);
-                        }
-                        xb = 0;
-                        ent += ENT;
-                        orow += pitch_bytes;
-                    }
-                }
-            }
-        } else if (interior) {
-            // every unit is whole and lies in segment l0: the lean loop, rows outside, boxes inside
-            RowCtx<RMAX> c;
-            const int nbx = p.nbx;
-            const unsigned char* ent = tab0 + (size_t)row * ENT;
-            unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
-            const uint32_t lane_base = stage_s + lane * GB;
-            int u = u_begin;
-            while (u < u_end) {
-                load_entry<RMAX>(ent, c);
-                for (; xb < nbx && u < u_end; ++xb, ++u) {
-                    const uint32_t ubase = lane_base + xb * block_bytes;
-                    unsigned char* uout = orow + xb * box_payload;
-#pragma unroll
-                    for (int ch = 0; ch < CPB; ++ch)
-                        if (ch * 512 < box_payload)
-                            item_fast<EB, GB, RMAX, (RT >= 0)>(ubase + ch * 512, c, R, uout + ch * 512, pmask[ch]);
-                }
-                xb = 0;
-                ent += ENT;
-                orow += pitch_bytes;
-            }
-        } else {
-            // last tile of the rows, or a tile holding a segment boundary: element by element,
-            // except whole 128-bit groups that lie in one segment
-            for (int u = u_begin; u < u_end; ++u) {
-#pragma unroll 1
-                for (int ch = 0; ch < CPB; ++ch) {
-                    if (ch * 512 >= box_payload) continue;               // half-width boxes hold one item per row
-                    const int ib = xb * box_payload + ch * 512;          // byte offset of the item in the row
-                    const uint32_t ubase = stage_s + xb * block_bytes + ch * 512 + lane * GB;
-                    bool done = false;
-                    if (GB == 16) {
-                        const long long c0 = t0 + (ib + lane * 16) / EB;
-                        const bool whole = c0 + V <= p.width;
-                        const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
-                        if (whole && one_seg) {
-                            RowCtx<RMAX> cc;
-                            load_entry<RMAX>(tab0 + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
-                            item_fast<EB, GB, RMAX, (RT >= 0)>(
-                                ubase, cc, R, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
-                            done = true;
-                        }
-                    }
-                    if (!done) {
-#pragma unroll 1
-                        for (int i = 0; i < PIECES; ++i) {
-                            const int pin = ch * 512 + lane * GB + i * PSTRIDE;  // byte offset inside the box payload
-                            if (pin >= box_payload) continue;
-#pragma unroll 1
-                            for (int e = 0; e < EPP; ++e) {
-                                const long long col = t0 + (xb * box_payload + pin) / EB + e;
-                                if (col >= p.width) continue;
-                                const unsigned char* ent = tab0 + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
-                                const float* cf = reinterpret_cast<const float*>(ent);       // pairs
-                                const int* po = reinterpret_cast<const int*>(cf + 2 * (RMAX + 1));
-                                const unsigned char* eb = stage + xb * block_bytes + pin + e * EB;
-                                float acc = __fmul_rn(cf[0], ElemOps<EB>::load(eb + po[0]));
-                                for (int r = 1; r <= R; ++r)
-                                    acc = fmaf(cf[2 * r], ElemOps<EB>::load(eb + po[r]), acc);
-                                ElemOps<EB>::store(p.out + (size_t)row * pitch_bytes + (size_t)col * EB, acc);
-                            }
-                        }
-                    }
-                }
-                if (++xb == p.nbx) { xb = 0; ++row; }
-            }
-        }
         // The fused step rewrote the stage with ordinary stores; the copy that refills it goes
         // through the asynchronous proxy, so the two are ordered by a proxy fence.
         if (SGD) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
     }
+}
+
+// ---------------------------------------------------------------- one tile per CTA
+// Short kernels (a few tiles per SM in all) spend much of their time filling and draining a
+// ring; here every tile is a CTA of its own and several CTAs share an SM.  All loads of the
+// first wave are in flight at once, a CTA leaves as soon as its tile is written, and the
+// hardware's block scheduler does what the tile dispenser does in k_staged.  One TMA load
+// (issued by warp 0), the coefficient table of the tile's two possible segments built
+// meanwhile, then the same per-warp aggregation as above.
+constexpr int kTileWarps = 4;
+constexpr int kTileThreads = 32 * kTileWarps;
+
+template <int EB, int GB, bool SGD, int RT>
+__global__ void __launch_bounds__(kTileThreads)
+k_tile(const AggParams p, const __grid_constant__ TileMaps maps) {
+    constexpr int RMAX = (RT >= 0) ? RT : (RT == -2 ? kStagedMaxR : kGenericR);
+    extern __shared__ __align__(128) unsigned char smem[];
+    StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int N = p.N, R = (RT >= 0) ? RT : p.R;
+    const int narr = SGD ? 2 : 1;
+    unsigned char* tab = smem + p.tab_off;                 // two slots: segments l0 and l0 + 1
+    unsigned char* stage = smem + p.stage_off;
+    const int block_bytes = N * p.row_bytes;
+    const uint32_t bar = smem_u32(&hdr->full[0]);
+    const long long tile = blockIdx.x;
+    const long long t0 = tile * (long long)p.T;
+    const int l0 = (int)((p.p_begin + t0) / p.L);
+    const long long bnd = (long long)(l0 + 1) * p.L - p.p_begin;   // local column where l0 + 1 starts
+
+    // lane of warp 0 -> one TMA box: (array a, x-box b, class j), as in k_staged
+    const int per_arr = p.nbx * p.m;
+    const int a = lane / per_arr, rem = lane - a * per_arr;
+    const int b = rem / p.m, j = rem - b * p.m;
+    const bool issuer = warp == 0 && lane < narr * per_arr && j < N;
+    int class_base = 0;
+    for (int q = 0; q < j; ++q) class_base += (N - q + p.m - 1) / p.m;
+    const CUtensorMap* my_map = &maps.map[issuer ? a : 0][issuer ? j : 0];
+    if (issuer) asm volatile("prefetch.tensormap [%0];" ::"l"(my_map) : "memory");
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_arrive_expect_tx(bar, p.stage_bytes);
+    }
+    // A CTA of this kernel is small, so under programmatic stream serialization it becomes
+    // resident while the preceding kernel still runs.  Its tile is asked into L2 right away:
+    // a prefetch has no architectural effect (if the preceding kernel is still writing these
+    // lines, L2 keeps them coherent and the load below sees the final values), but the read
+    // from HBM then overlaps the preceding kernel's tail instead of following it.
+    const int box_x = (int)(t0 + (long long)b * (p.T / p.nbx));
+    if (issuer) tma_prefetch_2d(my_map, box_x, 0);
+    __syncthreads();
+    // everything above touched only this CTA's shared memory and the launch parameters (see
+    // k_staged on programmatic stream serialization)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (issuer)
+        tma_load_2d(smem_u32(stage) + (uint32_t)((a * p.nbx + b) * block_bytes + class_base * p.row_bytes), my_map,
+                    box_x, 0, bar);
+    // the second slot only where the tile reaches into segment l0 + 1
+    build_coef_table<EB, RMAX>(p, tab, R, l0, bnd < t0 + p.T ? 2 : 1, tid, kTileThreads);
+    __syncthreads();
+    if (!mbar_wait(bar, 0)) {
+        // give the copy one more bounded chance to land before the shared memory is released
+        staged_fail(8);
+        mbar_wait(bar, 0);
+        return;
+    }
+    if (SGD) {
+        sgd_step_in_place(stage, p.nbx * block_bytes, p.lr, tid, kTileThreads);
+        __syncthreads();
+    }
+    const WarpShare<EB, GB> ws(p, warp, kTileWarps, lane);
+    aggregate_tile<EB, GB, RT>(p, ws, stage, smem_u32(stage), tab, tile, bnd, lane);
 }
 
 }  // namespace combo

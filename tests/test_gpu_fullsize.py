@@ -69,7 +69,7 @@ def test_workload_full_size_sampled(name):
         else:
             combo.combo_segment_aggregate(cur, nxt, weights, idx, wl.N, wl.P, wl.S, wl.R)
         torch.cuda.synchronize()
-        assert combo.combo_last_kernel_path() == combo.PATH_STAGED
+        assert combo.combo_last_kernel_path() in (combo.PATH_STAGED, combo.PATH_TILE)
         for sp in spans:
             a, b = sp
             got = to_bits(nxt[:, a:b])

@@ -1,4 +1,4 @@
-"""Randomised shapes: both aggregation kernels against the oracle and each other."""
+"""Randomised shapes: the aggregation kernels against the oracle and each other."""
 import numpy as np
 import pytest
 import torch
@@ -31,6 +31,8 @@ def test_random_shapes(seed):
     a, _ = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_STAGED)
     b, _ = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_DIRECT)
     assert torch.equal(a, b), (N, P, S, R, dtype, fused)
+    c, _ = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_TILE)
+    assert torch.equal(a, c), (N, P, S, R, dtype, fused)
     lo, hi = 0, min(P, 3000)
     mid = P // 2
     for (c0, c1) in ((lo, hi), (max(mid - 1500, 0), min(mid + 1500, P)), (max(P - 3000, 0), P)):
@@ -61,6 +63,10 @@ def test_random_long_rows(seed):
     assert used == combo.PATH_STAGED, (N, P, S, R, dtype, fused)
     b, _ = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_DIRECT)
     assert torch.equal(a, b), (N, P, S, R, dtype, fused)
+    c, used_c = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_TILE)
+    assert torch.equal(a, c), (N, P, S, R, dtype, fused)
+    if (P * x.element_size()) % 16 == 0:
+        assert used_c == combo.PATH_TILE
     L = -(-P // S)
     windows = [(0, 2000), (max(P - 2000, 0), P)]
     if S > 1:

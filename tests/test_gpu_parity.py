@@ -134,6 +134,47 @@ def test_aggregate_medium_both_kernels(N, P, S, R, dtype, weighted, path):
         check_against_oracle(x, out, idx_np, S, R, weights=weights, grads=grads, lr=0.01)
 
 
+@pytest.mark.parametrize("N,P,S,R,dtype,weighted", MEDIUM)
+def test_aggregate_medium_one_tile_per_cta(N, P, S, R, dtype, weighted):
+    # the kernel for short inputs (one tile per CTA); rows whose 16-byte phases differ and
+    # R > 16 fall back to the other kernels, everything else must really run on it
+    x, grads, counts = _inputs(N, P, dtype, 17 * N + P % 1000)
+    weights = counts if weighted else None
+    idx_np = oracle.select_peers(1, 2, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV) if R > 0 else None
+    out, used = gpu_aggregate(x, idx, S, R, weights=weights, path=combo.PATH_TILE)
+    if (P * x.element_size()) % 16 == 0 and R <= 16:
+        assert used == combo.PATH_TILE
+    check_against_oracle(x, out, idx_np, S, R, weights=weights)
+    if dtype == torch.float32:
+        out, used = gpu_aggregate(x, idx, S, R, weights=weights, grads=grads, lr=0.01, path=combo.PATH_TILE)
+        check_against_oracle(x, out, idx_np, S, R, weights=weights, grads=grads, lr=0.01)
+
+
+@pytest.mark.parametrize("tile", [256, 512, 1024, 2048])
+def test_one_tile_per_cta_tile_widths(tile):
+    # several boxes per tile, ragged last tile, segment boundaries inside tiles
+    N, P, S, R = 8, 100_004, 7, 3
+    x, grads, counts = _inputs(N, P, torch.float32, 5)
+    idx_np = oracle.select_peers(9, 0, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    combo.combo_set_tuning(tile, 0)
+    try:
+        out, used = gpu_aggregate(x, idx, S, R, weights=counts, path=combo.PATH_TILE)
+        assert used == combo.PATH_TILE
+        check_against_oracle(x, out, idx_np, S, R, weights=counts)
+        out, used = gpu_aggregate(x, idx, S, R, grads=grads, lr=0.01, path=combo.PATH_TILE)
+        if tile <= 1024:
+            assert used == combo.PATH_TILE
+        check_against_oracle(x, out, idx_np, S, R, grads=grads, lr=0.01)
+        xb = x[:, :100_000].contiguous().to(torch.bfloat16)      # a 16-byte multiple per row in bf16 too
+        outb, used = gpu_aggregate(xb, idx, S, R, path=combo.PATH_TILE)
+        assert used == combo.PATH_TILE
+        check_against_oracle(xb, outb, idx_np, S, R)
+    finally:
+        combo.combo_set_tuning(0, 0)
+
+
 @pytest.mark.parametrize("tile,stages", [(256, 2), (256, 8), (512, 3), (768, 2), (1024, 3), (0, 0)])
 def test_staged_tile_shapes(tile, stages):
     # many tiles per CTA, several TMA boxes per tile, ragged last tile, segment
