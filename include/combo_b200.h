@@ -10,13 +10,19 @@
  * and the library allocates nothing.
  *
  * Library-owned device memory: a 4-byte status word (combo_device_status) and
- * a ring of 256 tile dispensers, 16 bytes each, of which every launch of the
- * staged aggregation kernel takes the next one (its CTAs draw their tiles
- * from it and the last one to leave clears it).  Launches that are in flight
- * at the same time therefore hold different dispensers, as long as fewer
- * than 256 launches separate them; a CUDA graph keeps the dispensers its
- * kernels were captured with, so two DIFFERENT graphs captured a multiple of
- * 256 launches apart must not run concurrently.
+ * a ring of 256 tile dispensers, 16 bytes each.  Every launch of the staged
+ * aggregation kernel with persistent CTAs takes the next dispenser (its CTAs
+ * draw their tiles from it and the last one to leave clears it): ordinary
+ * launches cycle through one half of the ring, launches that are being
+ * captured into a CUDA graph through the other half.  Ordinary launches in
+ * flight at the same time therefore hold different dispensers as long as
+ * fewer than 128 staged launches separate them, and a graph replay never
+ * shares one with ordinary launches running beside it.  A graph keeps the
+ * dispensers it was captured with: two replays (of one graph or of different
+ * ones) whose staged kernels could run at the same time must not hold the
+ * same dispenser -- do not run a graph concurrently with itself, nor with a
+ * graph captured a multiple of 128 staged launches before or after it.
+ * Sharing a dispenser loses or repeats tiles (wrong output, no fault).
  *
  * Notation follows the paper: n = N workers, S segments, R model replicas,
  * |D_j| dataset size of worker j, P_l the set of workers providing segment l.
@@ -187,14 +193,15 @@ combo_status combo_check_rows(const void* const* d_rows, int N, void* stream, in
  *
  * combo_segment_aggregate_members: Eq. 3 with the provider set
  *   P_l(w) = ({w} unless w is a newcomer) U { idx[w][l][r] : idx[w][l][r] >= 0 }.
- * A new worker "pulls the segments and aggregates them as normal only without
- * its local model", so its own row is never read; a negative idx entry is a
- * pull that found no online peer.  A worker left with no provider (an offline
+ * A newcomer has no model of its own yet: it aggregates the segments it
+ * pulled without an own term (Section 4.2), so its row is never read; a
+ * negative idx entry is a pull that found no online peer.  A worker left with no provider (an offline
  * worker's -1 rows) keeps its own values.  h_newcomer: HOST array of N bytes,
  * non-zero = newcomer, or NULL.  Same arithmetic and order as
  * combo_segment_aggregate (providers in the order self, peers ascending); all
- * entry points above accept negative idx entries in the same way.  Rows that are
- * read must hold finite values.
+ * entry points above accept negative idx entries in the same way (the
+ * worker-sharded call too; it has no newcomer flags).  Rows that are read must
+ * hold finite values.
  */
 combo_status combo_select_peers_online(uint64_t seed, uint32_t round, int N, int S, int R,
                                        const uint8_t* h_online, int32_t* idx_out, void* stream);
@@ -322,6 +329,30 @@ void combo_set_tuning(int tile_elems, int stages);
  * hides is launch latency and set-up between back-to-back rounds (Section
  * 4.1: one synchronization per iteration).  0 = ordinary launches. */
 void combo_set_launch_overlap(int on);
+
+/* Widest column range a single aggregation launch takes (the staged kernels
+ * address columns with signed 32-bit copy coordinates).  Wider inputs are cut
+ * into column shards of this many columns inside the call, one launch each;
+ * Eq. 3 couples workers only at equal column, so the result is the same. */
+int64_t combo_max_launch_columns(void);
+
+/* Expert / test knob, this thread only: cut inputs into shards of `columns`
+ * columns instead (rounded down to a multiple of 64; 0 or out of range
+ * restores combo_max_launch_columns()). */
+void combo_set_launch_columns(int64_t columns);
+
+/*
+ * Self-check of the time-out path (no counterpart in the paper).  Every wait
+ * inside the kernels is bounded; a wait that runs out sets the device status
+ * word and the kernel returns, which combo_device_status() then reports as
+ * COMBO_ERR_DEVICE_TIMEOUT.  This call enqueues a one-warp kernel that waits,
+ * with a cap of a thousand polls, on a barrier of its own that nothing ever
+ * signals, and reports in the same way: after it, combo_device_status()
+ * returns COMBO_ERR_DEVICE_TIMEOUT once (site 99 in combo_last_cuda_error())
+ * and COMBO_OK afterwards.  It touches no product kernel and leaves nothing
+ * armed; the device and the context stay usable.
+ */
+combo_status combo_debug_dead_wait(void* stream);
 
 const char* combo_status_string(combo_status status);
 const char* combo_last_cuda_error(void);

@@ -9,4 +9,5 @@ from .binding import (ComboError, combo_aggregation_divergence, combo_aggregatio
                       combo_select_peers_online,
                       combo_select_peers_default_stream, combo_set_kernel_path, combo_set_launch_overlap,
                       combo_set_tuning,
-                      combo_validate_idx, combo_version, load)
+                      combo_validate_idx, combo_version, load, combo_max_launch_columns,
+                      combo_set_launch_columns, combo_debug_dead_wait)

@@ -55,6 +55,7 @@ def load():
                              vp, vp, vp, vp],
         "combo_aggregation_divergence": [vp, vp, i32, vp, i32, i64, vp, vp, ctypes.c_size_t, vp],
         "combo_aggregation_divergence_noalloc": [vp, vp, i32, vp, i32, i64, vp, vp],
+        "combo_debug_dead_wait": [vp],
         "combo_device_status": [],
         "combo_last_kernel_path": [],
         "combo_version": [],
@@ -69,6 +70,10 @@ def load():
     lib.combo_set_kernel_path.restype = None
     lib.combo_set_tuning.argtypes = [i32, i32]
     lib.combo_set_tuning.restype = None
+    lib.combo_max_launch_columns.argtypes = []
+    lib.combo_max_launch_columns.restype = ctypes.c_int64
+    lib.combo_set_launch_columns.argtypes = [i64]
+    lib.combo_set_launch_columns.restype = None
     lib.combo_set_launch_overlap.argtypes = [i32]
     lib.combo_set_launch_overlap.restype = None
     lib.combo_status_string.argtypes = [i32]
@@ -243,6 +248,19 @@ def combo_set_tuning(tile_elems: int = 0, stages: int = 0) -> None:
 
 def combo_set_launch_overlap(on: bool = True) -> None:
     load().combo_set_launch_overlap(1 if on else 0)
+
+
+def combo_max_launch_columns() -> int:
+    return int(load().combo_max_launch_columns())
+
+
+def combo_set_launch_columns(columns: int = 0) -> None:
+    load().combo_set_launch_columns(columns)
+
+
+def combo_debug_dead_wait(stream=None) -> None:
+    """Enqueues the self-check kernel whose bounded wait runs out (see the header)."""
+    _check(load().combo_debug_dead_wait(_stream(stream)), "combo_debug_dead_wait")
 
 
 def combo_version() -> int:

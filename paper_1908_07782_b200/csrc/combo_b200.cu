@@ -75,9 +75,9 @@ inline unsigned round_up(unsigned v, unsigned q) { return (v + q - 1) / q * q; }
 // zero when idle (the kernel's last CTA resets it), so launches that overlap on the device
 // only need different slots: 256 of them cover any number of kernels that can be resident.
 combo::TileSlot* g_slot_base[64];
-unsigned g_slot_seq = 0;
+unsigned g_slot_seq[2] = {0, 0};      // [0] ordinary launches, [1] launches being captured into a graph
 
-combo_status next_tile_slot(combo::TileSlot** out) {
+combo_status next_tile_slot(combo::TileSlot** out, cudaStream_t st) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
@@ -88,8 +88,15 @@ combo_status next_tile_slot(combo::TileSlot** out) {
         if (e != cudaSuccess || !ptr) return cuda_fail(e, "cudaGetSymbolAddress(tile slots)");
         g_slot_base[dev] = ptr;
     }
-    const unsigned seq = __atomic_fetch_add(&g_slot_seq, 1u, __ATOMIC_RELAXED);
-    *out = g_slot_base[dev] + (seq % combo::kTileSlots);
+    // A graph keeps the slots its kernels were captured with for as long as it is replayed,
+    // while ordinary launches move on through the ring: the two kinds draw from separate
+    // halves, so that a replay running beside ordinary launches never meets them on a slot.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+    const int kind = cap == cudaStreamCaptureStatusActive ? 1 : 0;
+    const unsigned half = combo::kTileSlots / 2;
+    const unsigned seq = __atomic_fetch_add(&g_slot_seq[kind], 1u, __ATOMIC_RELAXED);
+    *out = g_slot_base[dev] + kind * half + (seq % half);
     return COMBO_OK;
 }
 
@@ -447,6 +454,7 @@ cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo
 // widest column range one launch takes: a multiple of 64 elements (shards start on 16-byte
 // boundaries) that keeps every TMA coordinate, box width included, below 2^31
 constexpr long long kMaxShardColumns = 1LL << 30;
+thread_local long long t_shard_columns = kMaxShardColumns;
 
 combo_status aggregate_cols(const void* in, const void* grads, float lr, void* out, int EB,
                             const float* weights, const int32_t* idx, int N, long long P_total, int S, int R,
@@ -466,9 +474,9 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
 
     // The staged kernels address columns with signed 32-bit TMA coordinates.  Wider inputs are
     // cut into column shards, which Eq. 3 allows (workers are coupled only at equal column).
-    if (width > kMaxShardColumns) {
-        for (long long c0 = 0; c0 < width; c0 += kMaxShardColumns) {
-            const long long w = width - c0 < kMaxShardColumns ? width - c0 : kMaxShardColumns;
+    if (width > t_shard_columns) {
+        for (long long c0 = 0; c0 < width; c0 += t_shard_columns) {
+            const long long w = width - c0 < t_shard_columns ? width - c0 : t_shard_columns;
             combo_status rcs = aggregate_cols(static_cast<const char*>(in) + c0 * EB,
                                               grads ? static_cast<const char*>(grads) + c0 * EB : nullptr, lr,
                                               static_cast<char*>(out) + c0 * EB, EB, weights, idx, N, P_total, S, R,
@@ -520,7 +528,7 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
         combo::TileMaps maps;
         StagedPlan plan = plan_staged(p, maps, EB, sgd, *dev);
         if (plan.ok) {
-            rc = next_tile_slot(&p.sched);
+            rc = next_tile_slot(&p.sched, st);
             if (rc != COMBO_OK) return rc;
             cudaError_t e = launch_staged(p, maps, plan, EB, sgd, st);
             if (e != cudaSuccess) return cuda_fail(e, "staged aggregation launch");
@@ -1025,6 +1033,23 @@ void combo_set_tuning(int tile_elems, int stages) {
 }
 
 void combo_set_launch_overlap(int on) { t_overlap = on ? 1 : 0; }
+
+int64_t combo_max_launch_columns(void) { return kMaxShardColumns; }
+
+void combo_set_launch_columns(int64_t columns) {
+    long long c = columns / 64 * 64;
+    t_shard_columns = (c < 64 || c > kMaxShardColumns) ? kMaxShardColumns : c;
+}
+
+combo_status combo_debug_dead_wait(void* stream) {
+    DeviceInfo* dev = nullptr;
+    combo_status rc = device_info(&dev);
+    if (rc != COMBO_OK) return rc;
+    combo::k_debug_dead_wait<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "debug wait launch");
+    return COMBO_OK;
+}
 
 const char* combo_status_string(combo_status status) {
     switch (status) {

@@ -42,9 +42,12 @@ __global__ void __launch_bounds__(256) k_pull_aggregate(const PullParams p) {
         const long long hi = (c0 + V > p.P) ? p.P : c0 + V;
         const long long l_lo = c0 / p.L, l_hi = (hi - 1) / p.L;
         if (hi - c0 == V && l_lo == l_hi) {
+            // providers: the worker itself, then its peers ascending; a negative entry is a pull
+            // that found no online peer (Section 4.2) and is skipped
             const int32_t* peers = my_idx + (size_t)l_lo * R;
             float den = p.weights ? p.weights[w] : 1.0f;
-            for (int r = 0; r < R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+            for (int r = 0; r < R; ++r)
+                if (peers[r] >= 0) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
             float acc[V], x[V];
             GroupLoad<EB, 16>::run(rows[w] + (size_t)c0 * EB, x);
             float c = __fdiv_rn(p.weights ? p.weights[w] : 1.0f, den);
@@ -52,6 +55,7 @@ __global__ void __launch_bounds__(256) k_pull_aggregate(const PullParams p) {
             for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(c, x[i]);
             for (int r = 0; r < R; ++r) {
                 const int k = peers[r];
+                if (k < 0) continue;
                 GroupLoad<EB, 16>::run(rows[k] + (size_t)c0 * EB, x);
                 c = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
 #pragma unroll
@@ -63,11 +67,13 @@ __global__ void __launch_bounds__(256) k_pull_aggregate(const PullParams p) {
             for (long long col = c0; col < hi; ++col) {
                 const int32_t* peers = my_idx + (size_t)(col / p.L) * R;
                 float den = p.weights ? p.weights[w] : 1.0f;
-                for (int r = 0; r < R; ++r) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+                for (int r = 0; r < R; ++r)
+                    if (peers[r] >= 0) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
                 float acc = __fmul_rn(__fdiv_rn(p.weights ? p.weights[w] : 1.0f, den),
                                       ElemOps<EB>::load(rows[w] + (size_t)col * EB));
                 for (int r = 0; r < R; ++r) {
                     const int k = peers[r];
+                    if (k < 0) continue;
                     acc = fmaf(__fdiv_rn(p.weights ? p.weights[k] : 1.0f, den),
                                ElemOps<EB>::load(rows[k] + (size_t)col * EB), acc);
                 }

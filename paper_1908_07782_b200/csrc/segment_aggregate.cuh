@@ -528,6 +528,30 @@ __device__ __forceinline__ bool mbar_wait_brisk(uint32_t bar, uint32_t parity) {
     return false;
 }
 
+// Self-check of the give-up path every bounded wait shares: one warp waits, with a cap of a
+// thousand polls, on a barrier of its own that nothing ever arrives at, then reports through
+// the status word exactly as the aggregation kernels do and returns.  Nothing is left armed:
+// the barrier lives in this CTA's shared memory and no copy was started.
+constexpr int kDebugWaitSite = 99;
+__global__ void k_debug_dead_wait() {
+    __shared__ unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const uint32_t b = smem_u32(&bar);
+    uint32_t ok = 0;
+#pragma unroll 1
+    for (uint32_t it = 0; it < 1000u && !ok; ++it)
+        asm volatile(
+            "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+            : "=r"(ok)
+            : "r"(b), "r"(0u)
+            : "memory");
+    if (!ok && threadIdx.x == 0) staged_fail(kDebugWaitSite);
+}
+
 // Consumer-wide barrier with a bounded wait (all 16 consumer warps).
 __device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t& phase, int lane) {
     __syncwarp();

@@ -62,6 +62,18 @@ def pull_traffic(idx: np.ndarray, world: int, P: int, elem_bytes: int) -> np.nda
     return out
 
 
+def row_addresses(bases, N: int, pitch_bytes: int) -> list[int]:
+    """Address of every worker's row given each rank's buffer base (``bases[g]`` as rank g maps
+    it): worker w lives on owner_of(w), at local row w - (first worker of that rank)."""
+    world = len(bases)
+    addr = []
+    for w in range(N):
+        o = owner_of(w, world, N)
+        first, _ = worker_range(o, world, N)
+        addr.append(int(bases[o]) + (w - first) * pitch_bytes)
+    return addr
+
+
 class ShardedFederation:
     """The hosted workers of this rank and the rounds over them.  Needs an initialised
     NCCL process group (one rank per GPU of the node) and the CUDA library."""
@@ -92,12 +104,7 @@ class ShardedFederation:
             h = symm_mem.rendezvous(t, self.group)
             self.bufs.append(t)
             self.handles.append(h)
-            bases = [int(b) for b in h.buffer_ptrs]
-            addr = []
-            for w in range(N):
-                o = owner_of(w, self.world, N)
-                first, _ = worker_range(o, self.world, N)
-                addr.append(bases[o] + (w - first) * self.pitch * self.elem_bytes)
+            addr = row_addresses([int(b) for b in h.buffer_ptrs], N, self.pitch * self.elem_bytes)
             self.row_tables.append(torch.tensor(addr, dtype=torch.int64, device=self.dev))
         self.weights = weights
         self.idx = torch.empty((N, S, max(R, 1)), dtype=torch.int32, device=self.dev)

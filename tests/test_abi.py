@@ -48,6 +48,18 @@ def test_host_side_argument_checks_need_no_device():
     assert lib.combo_segment_aggregate(a, a + 32, None, None, 2, 4, 1, 1, None) == 1  # idx missing
 
 
+def test_launch_column_limit_keeps_copy_coordinates_in_int32():
+    # the staged kernels pass column numbers to the copy engine as signed 32-bit values: the
+    # widest range one launch takes, plus the widest box (256 columns), must stay below 2^31,
+    # and shards must start on 16-byte boundaries for both element sizes
+    lim = combo.combo_max_launch_columns()
+    assert lim + 256 < 2 ** 31 and lim % 64 == 0 and lim >= 2 ** 28
+    # a 2^31-column row (8 GB in binary32) is therefore cut into several launches
+    assert -(-(2 ** 31) // lim) >= 2
+    combo.combo_set_launch_columns(100_000)      # rounded down to a multiple of 64; no device needed
+    combo.combo_set_launch_columns(0)
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     from paper_1908_07782_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)

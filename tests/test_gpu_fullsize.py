@@ -6,7 +6,10 @@ Eq. 3 couples workers only at equal column, so the oracle can be evaluated on
 any set of columns on its own, round after round: the sampled slabs are copied
 to the host before each launch and evolved there by the oracle.  Samples cover
 every segment boundary, the first and last columns, tile edges and a few
-random places."""
+random places.  In addition, where device memory allows, every round is repeated with the
+direct-gather kernel (itself pinned to the oracle on slabs of every size) into a third buffer
+and the two outputs are compared over the WHOLE array, bit for bit: a tile handed to the wrong
+stage at full size would show there even if it missed every sampled span."""
 import numpy as np
 import pytest
 import torch
@@ -44,10 +47,12 @@ def test_workload_full_size_sampled(name):
     need = wl.N * wl.P * (2 * e + (4 if wl.fused_sgd else 0)) * 1.1 + 2e9
     if free < need:
         pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
+    whole_array = free >= need + wl.N * wl.P * e * 1.05      # room for the direct kernel's output
     rng = np.random.default_rng(7)
     spans = sample_ranges(wl, rng)
     cur = synth.make_params(wl, DEV)
     nxt = torch.empty_like(cur)
+    third = torch.empty_like(cur) if whole_array else None
     weights = synth.make_weights(wl, DEV)
     wn = weights.cpu().numpy() if weights is not None else None
     idx = torch.empty((wl.N, wl.S, wl.R), dtype=torch.int32, device=DEV)
@@ -70,6 +75,20 @@ def test_workload_full_size_sampled(name):
             combo.combo_segment_aggregate(cur, nxt, weights, idx, wl.N, wl.P, wl.S, wl.R)
         torch.cuda.synchronize()
         assert combo.combo_last_kernel_path() in (combo.PATH_STAGED, combo.PATH_TILE)
+        if third is not None:
+            combo.combo_set_kernel_path(combo.PATH_DIRECT)
+            try:
+                if wl.dtype == "bf16":
+                    combo.combo_segment_aggregate_bf16(cur, third, weights, idx, wl.N, wl.P, wl.S, wl.R)
+                elif wl.fused_sgd:
+                    combo.combo_segment_aggregate_sgd(cur, grads, wl.lr, third, weights, idx, wl.N, wl.P, wl.S, wl.R)
+                else:
+                    combo.combo_segment_aggregate(cur, third, weights, idx, wl.N, wl.P, wl.S, wl.R)
+            finally:
+                combo.combo_set_kernel_path(combo.PATH_AUTO)
+            torch.cuda.synchronize()
+            assert combo.combo_last_kernel_path() == combo.PATH_DIRECT
+            assert torch.equal(nxt, third), (name, t, "staged and direct outputs differ somewhere in the array")
         for sp in spans:
             a, b = sp
             got = to_bits(nxt[:, a:b])

@@ -392,3 +392,48 @@ def test_largest_worker_count():
     with pytest.raises(combo.ComboError) as e:
         combo.combo_select_peers(7, 4, N + 1, S, R, torch.empty((N + 1, S, R), dtype=torch.int32, device=DEV))
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("path", [combo.PATH_AUTO, combo.PATH_STAGED, combo.PATH_DIRECT])
+def test_wide_inputs_run_as_column_shards(dtype, path):
+    # inputs wider than one launch takes are cut into column shards inside the call; with the
+    # limit lowered to 40,000 columns a 150,001-column input takes four launches, which must
+    # give the bits of the single launch (segment boundaries fall inside shards)
+    N, P, S, R = 9, 150_001, 4, 3
+    x, grads, counts = _inputs(N, P, dtype, 77)
+    idx_np = oracle.select_peers(2, 5, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    whole, _ = gpu_aggregate(x, idx, S, R, weights=counts, path=path)
+    combo.combo_set_launch_columns(40_000)
+    try:
+        cut, _ = gpu_aggregate(x, idx, S, R, weights=counts, path=path)
+        assert torch.equal(whole, cut)
+        check_against_oracle(x, cut, idx_np, S, R, weights=counts)
+        if dtype == torch.float32:
+            cut, _ = gpu_aggregate(x, idx, S, R, grads=grads, lr=0.01, path=path)
+            check_against_oracle(x, cut, idx_np, S, R, grads=grads, lr=0.01)
+    finally:
+        combo.combo_set_launch_columns(0)
+
+
+def test_a_wait_that_runs_out_is_reported_once():
+    # the give-up path of the bounded waits: a self-check kernel waits (a thousand polls) on a
+    # barrier nothing signals, sets the status word and returns; the context stays usable
+    combo.combo_device_status()
+    combo.combo_debug_dead_wait()
+    with pytest.raises(combo.ComboError) as e:
+        combo.combo_device_status()
+    assert e.value.status == 5
+    assert "site 99" in combo.load().combo_last_cuda_error().decode()
+    combo.combo_device_status()                     # cleared: reported once
+    # and the library works as before (the dispenser ring was cleaned with the status word)
+    N, P, S, R = 8, 300_000, 4, 2
+    x, _, counts = _inputs(N, P, torch.float32, 3)
+    idx_np = oracle.select_peers(1, 0, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    for path in (combo.PATH_STAGED, combo.PATH_TILE):
+        out, used = gpu_aggregate(x, idx, S, R, weights=counts, path=path)
+        assert used == path
+        check_against_oracle(x, out, idx_np, S, R, weights=counts)
+    combo.combo_device_status()

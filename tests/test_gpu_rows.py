@@ -9,7 +9,7 @@ import torch
 import oracle
 import paper_1908_07782_b200 as combo
 from paper_1908_07782_b200 import sharding
-from gpu_util import DEV, check_against_oracle
+from gpu_util import DEV, check_against_oracle, to_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -67,6 +67,39 @@ def test_rows_kernel_matches_oracle_and_dense_kernel(N, P, S, R, world, dtype, w
     torch.cuda.synchronize()
     assert torch.equal(union.view(torch.int16 if e == 2 else torch.int32),
                        ref.view(torch.int16 if e == 2 else torch.int32))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_rows_kernel_skips_pulls_that_found_no_peer(dtype):
+    # a table from the online sampler holds -1 rows for offline workers and -1 pulls
+    # (Section 4.2); the worker-sharded call must skip them like the dense kernels do
+    N, P, S, R = 10, 20_003, 4, 3
+    e = 4 if dtype == torch.float32 else 2
+    dense, rows, table = make_rows(N, P, dtype, seed=5)
+    w = torch.randint(500, 1501, (N,), generator=torch.Generator().manual_seed(3)).float().to(DEV)
+    active = np.ones(N, np.uint8)
+    active[[2, 7]] = 0
+    idx_np = oracle.select_peers_active(4, 1, N, S, R, active)
+    idx_np[0, 1, :] = -1                      # a segment left without any peer
+    idx_np[5, 2, 1] = -1                      # one pull of three missing
+    assert (idx_np[2] == -1).all()
+    idx = torch.from_numpy(idx_np).to(DEV)
+    vec = 16 // e
+    pitch = -(-P // vec) * vec
+    out = torch.empty(N, pitch, dtype=dtype, device=DEV)
+    combo.combo_segment_aggregate_rows(table, out, pitch, e, w, idx, N, P, S, R, 0, N)
+    torch.cuda.synchronize()
+    got = out[:, :P].contiguous()
+    want = oracle.segment_aggregate_members(to_bits(dense), idx_np, S, R, w.cpu().numpy(), np.zeros(N, np.uint8),
+                                            ordered=True)
+    assert (to_bits(got).view(np.uint8) == want.view(np.uint8)).all()
+    # offline workers keep their values
+    assert torch.equal(got[2], dense[2]) and torch.equal(got[7], dense[7])
+    ref = torch.empty_like(dense)
+    combo.combo_segment_aggregate_members(dense, ref, w, idx, None, N, P, S, R)
+    torch.cuda.synchronize()
+    assert torch.equal(got, ref)
+    combo.combo_device_status()
 
 
 def test_rows_argument_errors_and_pointer_check():

@@ -53,3 +53,22 @@ def test_one_rank_pulls_nothing_over_the_links():
     idx = oracle.select_peers(1, 0, 8, 4, 2)
     t = sharding.pull_traffic(idx, 1, 1_048_576, 4)
     assert t.shape == (1, 1) and t[0, 0] == 8 * 2 * 1_048_576 * 4
+
+
+def test_row_address_table_for_uneven_shares():
+    # every worker's address = its owner's base + its local row; checked against an
+    # independent walk over the ranks' ranges, for shares that differ by one
+    for N, world in ((7, 3), (10, 4), (64, 8), (9, 9), (13, 2), (5, 1)):
+        pitch_bytes = 4096 + 16 * world
+        bases = [(g + 1) * (1 << 32) + 256 * g for g in range(world)]
+        got = sharding.row_addresses(bases, N, pitch_bytes)
+        want = [None] * N
+        for g in range(world):
+            a, b = sharding.worker_range(g, world, N)
+            for local, w in enumerate(range(a, b)):
+                assert sharding.owner_of(w, world, N) == g
+                want[w] = bases[g] + local * pitch_bytes
+        assert got == want
+        assert len(set(got)) == N
+        sizes = [sharding.worker_range(g, world, N) for g in range(world)]
+        assert max(b - a for a, b in sizes) - min(b - a for a, b in sizes) <= 1

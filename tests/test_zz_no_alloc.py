@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_1908_07782_b200 as combo
 
 pytestmark = pytest.mark.gpu
@@ -34,6 +35,14 @@ def no_alloc(models, mean_of, weights):
     return rho.cpu().numpy()
 
 
+def oracle_rho(models, mean_of, weights):
+    """Eq. 7 by the CPU oracle on the same bytes."""
+    def bits(t):
+        t = t.detach().cpu().contiguous()
+        return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+    return oracle.divergence(bits(models), weights.cpu().numpy(), mean_of=None if mean_of is None else bits(mean_of))
+
+
 def inputs(N, P, dtype, seed):
     g = torch.Generator().manual_seed(seed)
     base = torch.randn(P, generator=g) * 0.05
@@ -53,9 +62,13 @@ def test_two_calls_in_a_row_match_the_scratch_taking_entry_point():
         got = no_alloc(x, y, w)
         assert (got >= 0).all()
         np.testing.assert_allclose(got, want, rtol=RTOL, atol=1e-12)
+        # and directly against the oracle, not only through the other entry point
+        np.testing.assert_allclose(got, oracle_rho(x, y, w), rtol=RTOL, atol=1e-12)
     # and once more on the fallback kernel (rows not 16-byte aligned), against its own mean
     x, _, w = inputs(9, 50_001, torch.float32, 3)
-    np.testing.assert_allclose(no_alloc(x, None, w), reference(x, None, w), rtol=RTOL, atol=1e-12)
+    got = no_alloc(x, None, w)
+    np.testing.assert_allclose(got, reference(x, None, w), rtol=RTOL, atol=1e-12)
+    np.testing.assert_allclose(got, oracle_rho(x, None, w), rtol=RTOL, atol=1e-12)
     combo.combo_device_status()
 
 
