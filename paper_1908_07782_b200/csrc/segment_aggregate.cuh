@@ -49,6 +49,10 @@ constexpr int kMaxClasses = 8;
 constexpr int kMaxBoxes = 8;              // x-boxes per tile
 constexpr uint32_t kWaitCap = 1u << 23;   // polls before a wait is declared dead
 constexpr uint32_t kWaitHintNs = 1000;    // time a single poll may stay suspended
+#ifndef COMBO_FAST_POLLS
+#define COMBO_FAST_POLLS 32
+#endif
+constexpr uint32_t kFastPolls = COMBO_FAST_POLLS;   // polls without a suspend hint before the hinted ones
 
 // Tile dispenser of one launch (global memory owned by the library, one of a ring of
 // slots).  `next` hands out tiles beyond the first one of each CTA; the last CTA to leave
@@ -440,7 +444,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
 #pragma unroll 1
-    for (uint32_t it = 0; it < 32; ++it) {
+    for (uint32_t it = 0; it < kFastPolls; ++it) {
         asm volatile(
             "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
             : "=r"(ok)
