@@ -62,7 +62,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graphs", action="store_true", help="never replay short steps from CUDA graphs")
-    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 direct gather, 2 staged")
+    ap.add_argument("--path", type=int, default=0,
+                    help="0 auto, 1 direct gather, 2 staged (persistent CTAs), 5 staged (one tile per CTA); "
+                         "with --op pull: 3 = nothing staged")
     ap.add_argument("--P", type=int, default=0, help="override the vector length (scaled-down runs)")
     ap.add_argument("--N", type=int, default=0, help="override the number of workers")
     ap.add_argument("--rounds", type=int, default=0, help="override the rounds per step")
@@ -316,6 +318,7 @@ def run_divergence(args, wl):
     else:
         combo.combo_segment_aggregate(x, out, weights, idx, wl.N, wl.P, wl.S, wl.R)
     combo.combo_set_tuning(args.tile, args.stages)
+    combo.combo_set_kernel_path(args.path)
     rho = torch.empty(wl.N, dtype=torch.float64, device=dev)
     scratch = torch.empty(combo.combo_divergence_scratch_bytes(wl.N) // 8, dtype=torch.float64, device=dev)
     stream = torch.cuda.current_stream()
@@ -372,6 +375,8 @@ def run_pull(args, wl):
     e = elem_bytes(wl)
     dtype = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     weights = synth.make_weights(wl, dev)
+    combo.combo_set_kernel_path(args.path)             # 3 forces the unstaged pull kernel
+    combo.combo_set_tuning(args.tile, args.stages)
     fed = sharding.ShardedFederation(wl.N, wl.P, wl.S, wl.R, dtype, weights=weights)
     x = synth.make_params(wl, dev)                     # same seeds on every rank: take the hosted rows
     fed.rows().copy_(x[fed.w_begin:fed.w_end])
@@ -396,17 +401,40 @@ def run_pull(args, wl):
     kernel_path = combo.combo_last_kernel_path()
     combo.combo_device_status()
 
+    # ---- the pull kernel alone (no barrier, no peer selection), for the roofline figure
+    nxt = 1 - fed.cur
+    def pull_only():
+        combo.combo_segment_aggregate_rows(fed.row_tables[fed.cur], fed.bufs[nxt], fed.pitch, fed.elem_bytes,
+                                           fed.weights, fed.idx, fed.N, fed.P, fed.S, fed.R, fed.w_begin,
+                                           fed.n_local, stream=stream)
+    for _ in range(3):
+        pull_only()
+    torch.cuda.synchronize()
+    dist.barrier()
+    ka = torch.cuda.Event(enable_timing=True)
+    kb = torch.cuda.Event(enable_timing=True)
+    ka.record(stream)
+    for _ in range(steps):
+        pull_only()
+    kb.record(stream)
+    torch.cuda.synchronize()
+    dist.barrier()
+    ms_k = torch.tensor([ka.elapsed_time(kb) / steps], device=dev, dtype=torch.float64)
+    dist.all_reduce(ms_k, op=dist.ReduceOp.MAX)
+    ms_k = float(ms_k)
+
     # ---- comparison arm: all-reduce of the same hosted vectors (the R = n-1 limit, Section 4.3)
     hosted = fed.rows()
     n_loc = hosted.shape[0]
     wsc = (weights[fed.w_begin:fed.w_end] if weights is not None
-           else torch.ones(n_loc, device=dev)).to(torch.float32)
-    acc = torch.empty(wl.P, dtype=torch.float32, device=dev)
+           else torch.ones(n_loc, device=dev)).to(hosted.dtype)
+    hosted_t = hosted.t()                              # [P][n_local] view
 
     def allreduce_step():
-        # local weighted sum of the hosted rows (fp32), then the sum over ranks
-        torch.matmul(wsc, hosted.to(torch.float32) if hosted.dtype != torch.float32 else hosted, out=acc)
+        # local weighted sum of the hosted rows (in the models' storage type), then the sum over ranks
+        acc = torch.mv(hosted_t, wsc)
         dist.all_reduce(acc, op=dist.ReduceOp.SUM)
+        return acc
 
     for _ in range(3):
         allreduce_step()
@@ -429,9 +457,14 @@ def run_pull(args, wl):
         traffic = sharding.pull_traffic(idx_np, world, wl.P, e)
         link = int((traffic.sum(axis=1) - np.diag(traffic)).max())      # most any one rank pulls over NVLink
         n_local_max = -(-wl.N // world)
-        alg = (wl.R + 2) * n_local_max * wl.P * e                        # per GPU: R+1 reads (no reuse), 1 write
+        if kernel_path == 4:
+            # staged: the hosted rows and every distinct pulled row read once, results written once
+            rows_local, rows_remote = sharding.distinct_rows_read(idx_np, world, 0, wl.P)
+            alg = int((rows_local + rows_remote + n_local_max) * wl.P * e)
+        else:
+            alg = (wl.R + 2) * n_local_max * wl.P * e                    # per GPU: R+1 reads (no reuse), 1 write
         peak, src = hbm_peak()
-        ach = alg / (ms * 1e-3) / 1e9
+        ach = alg / (ms_k * 1e-3) / 1e9
         line = {
             "metric": METRIC, "op": "worker_sharded_round", "value": wl.N * wl.P / (ms * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
@@ -442,13 +475,13 @@ def run_pull(args, wl):
             "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
                          "traffic": None, "peak_source": src,
                          "kernel": {3: "k_pull_aggregate", 4: "k_pull_staged"}.get(kernel_path, "?"),
-                         "algorithmic_bytes_per_launch": alg,
+                         "avg_launch_ms": ms_k, "algorithmic_bytes_per_launch": alg,
                          "nvlink_bytes_per_round_max_rank": link,
-                         "nvlink_gbs_max_rank": link / (ms * 1e-3) / 1e9},
-            "allreduce_arm": {"what": "weighted sum of the hosted rows + NCCL all-reduce (fp32 [P]) "
+                         "nvlink_gbs_max_rank": link / (ms_k * 1e-3) / 1e9},
+            "allreduce_arm": {"what": "weighted sum of the hosted rows + NCCL all-reduce of the [P] result "
                                       "-- the R = n-1 limit of Section 4.3",
                               "ms_per_step": ms_ar, "pull_round_over_allreduce": ms / ms_ar,
-                              "bytes_reduced_per_rank": 4 * wl.P},
+                              "bytes_reduced_per_rank": e * wl.P},
             "gpu_launches": 2 * steps,
         }
         print(json.dumps(line))

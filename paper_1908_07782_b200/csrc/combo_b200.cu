@@ -831,6 +831,73 @@ combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, 
     DeviceInfo* dev = nullptr;
     combo_status rc = device_info(&dev);
     if (rc != COMBO_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long L = (P + S - 1) / S;
+
+    // Staged form: the distinct rows a column tile needs are brought into shared memory once.
+    // A stage must hold the hosted rows and everything they can pull for up to two segments.
+    if (t_force_path != 3 && N <= combo::kPullMaxN && R <= combo::kStagedMaxR && (long long)n_local * P >= (1 << 16)) {
+        long long d_max = (long long)n_local * (1 + 2 * R);
+        if (d_max > N) d_max = N;
+        const int rt = ((R >= 1 && R <= 4) || R == 8) ? R : (R > combo::kGenericR ? -2 : -1);
+        const int rmax = rt >= 0 ? rt : (rt == -2 ? combo::kStagedMaxR : combo::kGenericR);
+        combo::PullStagedParams q;
+        memset(&q, 0, sizeof(q));
+        q.ptr_off = 0;
+        q.slot_off = round_up((unsigned)N * 8u, 128);
+        q.list_off = q.slot_off + round_up((unsigned)N * 2u, 128);
+        q.tab_off = q.list_off + round_up((unsigned)d_max * 2u, 128);
+        q.stage_off = q.tab_off + round_up(2u * (unsigned)n_local * (unsigned)combo::table_entry_bytes(rmax), 128);
+        int T = 0;
+        for (int t = 256; t >= (elem_bytes == 4 ? 128 : 256); t >>= 1) {
+            const long long need = (long long)q.stage_off + 3LL * d_max * t * elem_bytes + 16;
+            if (need <= dev->smem_optin && t <= L) { T = t; break; }
+        }
+        if (T > 0) {
+            q.rows = d_rows;
+            q.out = static_cast<unsigned char*>(out);
+            q.weights = weights;
+            q.idx = idx;
+            q.P = P;
+            q.L = L;
+            q.out_pitch = out_pitch;
+            q.N = N; q.S = S; q.R = R;
+            q.w_begin = w_begin;
+            q.n_local = n_local;
+            q.T = T;
+            q.row_bytes = T * elem_bytes;
+            q.d_max = (int)d_max;
+            q.stage_bytes = (unsigned)(d_max * T * elem_bytes);
+            q.n_tiles = (P + T - 1) / T;
+            // about 64 KB of loads in flight beside the tile being consumed (measured: 3 stages of 32 KB beat 5), at least three stages
+            int stages = 1 + (int)((64 * 1024 + q.stage_bytes - 1) / q.stage_bytes);
+            const int fit = (int)(((long long)dev->smem_optin - q.stage_off - 16) / q.stage_bytes);
+            if (t_stages >= 3) stages = t_stages;
+            if (stages > 8) stages = 8;
+            if (stages > fit) stages = fit;
+            if (stages < 3) stages = 3;
+            q.stages = stages;
+            const size_t smem = (size_t)q.stage_off + (size_t)stages * (size_t)q.stage_bytes + 16;
+            const int grid = (int)(q.n_tiles < dev->sms ? q.n_tiles : dev->sms);
+            cudaError_t e = cudaErrorInvalidValue;
+#define COMBO_PULL_LAUNCH(EBV, RTV)                                                                              \
+    if (elem_bytes == EBV && rt == RTV) {                                                                        \
+        e = cudaFuncSetAttribute(combo::k_pull_staged<EBV, RTV>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+                                 (int)smem);                                                                     \
+        if (e == cudaSuccess) combo::k_pull_staged<EBV, RTV><<<grid, combo::kPullThreads, smem, st>>>(q);        \
+    }
+            COMBO_PULL_LAUNCH(4, 1) COMBO_PULL_LAUNCH(4, 2) COMBO_PULL_LAUNCH(4, 3) COMBO_PULL_LAUNCH(4, 4)
+            COMBO_PULL_LAUNCH(4, 8) COMBO_PULL_LAUNCH(4, -1) COMBO_PULL_LAUNCH(4, -2)
+            COMBO_PULL_LAUNCH(2, 1) COMBO_PULL_LAUNCH(2, 2) COMBO_PULL_LAUNCH(2, 3) COMBO_PULL_LAUNCH(2, 4)
+            COMBO_PULL_LAUNCH(2, 8) COMBO_PULL_LAUNCH(2, -1) COMBO_PULL_LAUNCH(2, -2)
+#undef COMBO_PULL_LAUNCH
+            if (e == cudaSuccess) e = cudaGetLastError();
+            if (e != cudaSuccess) return cuda_fail(e, "staged pull aggregation launch");
+            t_last_path = 4;
+            return COMBO_OK;
+        }
+    }
+
     combo::PullParams p;
     memset(&p, 0, sizeof(p));
     p.rows = d_rows;
@@ -838,7 +905,7 @@ combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, 
     p.weights = weights;
     p.idx = idx;
     p.P = P;
-    p.L = (P + S - 1) / S;
+    p.L = L;
     p.out_pitch = out_pitch;
     p.N = N; p.S = S; p.R = R;
     p.w_begin = w_begin;
@@ -852,7 +919,6 @@ combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, 
     if (bx > cap) bx = cap;
     const dim3 grid((unsigned)bx, (unsigned)n_local);
     const size_t smem = (size_t)N * sizeof(void*);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaSuccess;
     if (elem_bytes == 4) {
         if (smem > 48 * 1024) e = cudaFuncSetAttribute(combo::k_pull_aggregate<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -1025,7 +1091,7 @@ combo_status combo_device_status(void) {
 
 int combo_last_kernel_path(void) { return t_last_path; }
 
-void combo_set_kernel_path(int path) { t_force_path = (path == 1 || path == 2 || path == 5) ? path : 0; }
+void combo_set_kernel_path(int path) { t_force_path = (path == 1 || path == 2 || path == 3 || path == 5) ? path : 0; }
 
 void combo_set_tuning(int tile_elems, int stages) {
     t_tile = tile_elems > 0 ? tile_elems : 0;

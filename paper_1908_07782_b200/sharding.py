@@ -62,6 +62,25 @@ def pull_traffic(idx: np.ndarray, world: int, P: int, elem_bytes: int) -> np.nda
     return out
 
 
+def distinct_rows_read(idx: np.ndarray, world: int, rank: int, P: int) -> tuple[float, float]:
+    """What the staged worker-sharded kernel reads on ``rank``, in units of whole rows (P
+    elements): (local, remote).  Per segment it brings the hosted workers' own rows and every
+    DISTINCT other row some hosted worker pulls -- a (peer, segment) that several hosted
+    workers pull is fetched once -- so the figures are sums over segments of distinct counts
+    weighted by the segment's share of the vector."""
+    N, S, R = idx.shape
+    a, b = worker_range(rank, world, N)
+    seg = segment_lengths(P, S).astype(np.float64) / float(P)
+    local = remote = 0.0
+    for l in range(S):
+        pulled = set(int(k) for k in idx[a:b, l, :].ravel() if k >= 0)
+        others = [k for k in pulled if not (a <= k < b)]
+        n_remote = sum(1 for k in others if owner_of(k, world, N) != rank)
+        local += seg[l] * ((b - a) + len(others) - n_remote)
+        remote += seg[l] * n_remote
+    return local, remote
+
+
 def row_addresses(bases, N: int, pitch_bytes: int) -> list[int]:
     """Address of every worker's row given each rank's buffer base (``bases[g]`` as rank g maps
     it): worker w lives on owner_of(w), at local row w - (first worker of that rank)."""

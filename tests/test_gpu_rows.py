@@ -32,8 +32,13 @@ def make_rows(N, P, dtype, seed):
     (9, 1_003, 9, 8, 3, torch.bfloat16, True),        # R = N - 1: every worker pulls from all others
     (5, 300, 300, 1, 5, torch.float32, False),        # one-element segments
     (6, 4_096, 1, 0, 2, torch.float32, False),        # R = 0: identity
+    (64, 120_008, 10, 4, 8, torch.float32, False),    # 8 hosted workers of 64: many shared pulls
+    (128, 30_008, 16, 4, 4, torch.bfloat16, True),
+    (30, 100_000, 10, 12, 3, torch.float32, True),    # the wide kernel (R > 8)
+    (12, 70_000, 5, 6, 2, torch.float32, False),      # the unspecialised one
 ])
-def test_rows_kernel_matches_oracle_and_dense_kernel(N, P, S, R, world, dtype, weighted):
+@pytest.mark.parametrize("path", [0, 3])
+def test_rows_kernel_matches_oracle_and_dense_kernel(N, P, S, R, world, dtype, weighted, path):
     e = 4 if dtype == torch.float32 else 2
     dense, rows, table = make_rows(N, P, dtype, seed=N * 1000 + S)
     w = None
@@ -50,9 +55,14 @@ def test_rows_kernel_matches_oracle_and_dense_kernel(N, P, S, R, world, dtype, w
         guard = 64
         buf = torch.full(((b - a) * pitch + 2 * guard,), 7.0, dtype=dtype, device=DEV)
         out = buf[guard:guard + (b - a) * pitch].view(b - a, pitch)
-        combo.combo_segment_aggregate_rows(table, out, pitch, e, w, idx, N, P, S, R, a, b - a)
+        combo.combo_set_kernel_path(path)          # 3: nothing staged; 0: staged where the tile's rows fit
+        try:
+            combo.combo_segment_aggregate_rows(table, out, pitch, e, w, idx, N, P, S, R, a, b - a)
+        finally:
+            combo.combo_set_kernel_path(0)
         torch.cuda.synchronize()
-        assert combo.combo_last_kernel_path() == 3
+        staged_expected = path == 0 and (b - a) * P >= 65536
+        assert combo.combo_last_kernel_path() == (4 if staged_expected else 3)
         assert (buf[:guard] == 7.0).all() and (buf[guard + (b - a) * pitch:] == 7.0).all()
         if pitch > P:
             assert (out[:, P:] == 7.0).all(), "write into the row padding"
@@ -67,6 +77,7 @@ def test_rows_kernel_matches_oracle_and_dense_kernel(N, P, S, R, world, dtype, w
     torch.cuda.synchronize()
     assert torch.equal(union.view(torch.int16 if e == 2 else torch.int32),
                        ref.view(torch.int16 if e == 2 else torch.int32))
+    combo.combo_device_status()
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])

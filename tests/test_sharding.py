@@ -72,3 +72,21 @@ def test_row_address_table_for_uneven_shares():
         assert len(set(got)) == N
         sizes = [sharding.worker_range(g, world, N) for g in range(world)]
         assert max(b - a for a, b in sizes) - min(b - a for a, b in sizes) <= 1
+
+
+def test_distinct_rows_read_counts_shared_pulls_once():
+    # two hosted workers that pull the same (peer, segment) share one copy; a hosted worker
+    # pulled by another hosted worker costs nothing extra
+    N, S, R, P, world = 6, 2, 2, 1000, 3
+    idx = np.array([[[2, 4], [1, 5]], [[2, 4], [0, 3]], [[0, 1], [0, 1]], [[0, 1], [0, 1]],
+                    [[0, 1], [0, 1]], [[0, 1], [0, 1]]], dtype=np.int32)
+    local, remote = sharding.distinct_rows_read(idx, world, 0, P)       # rank 0 hosts workers 0, 1
+    # segment 0: pulled {2, 4} (both remote, shared by workers 0 and 1) -> 2 hosted + 2 remote
+    # segment 1: worker 0 pulls {1, 5}, worker 1 pulls {0, 3}: 1 and 0 are hosted -> remote {3, 5}
+    assert local == pytest.approx(2.0) and remote == pytest.approx(2.0)
+    # against the per-pull count of the paper: 2 workers x 2 pulls = 4 rows' worth per segment
+    t = sharding.pull_traffic(idx, world, P, 4)
+    assert t[0].sum() == 4 * 2 * (P // S) * 4
+    # one rank hosting everybody reads every row once
+    local, remote = sharding.distinct_rows_read(idx, 1, 0, P)
+    assert remote == 0.0 and local == pytest.approx(6.0)
