@@ -309,9 +309,13 @@ combo_status combo_device_status(void);
 int combo_last_kernel_path(void);
 
 /* Forces a path for the following calls on this thread: 0 automatic (default),
- * 1 direct gather, 2 staged with persistent CTAs (falls back to direct where
+ * 1 direct gather (blocks taken worker-fastest, so that the gather's re-reads
+ * are served by L2), 2 staged with persistent CTAs (falls back to direct where
  * staging cannot apply), 5 staged with one tile per CTA (falls back to 2 where
- * rows differ in their 16-byte phase or a tile does not fit). */
+ * rows differ in their 16-byte phase or a tile does not fit), 6 direct gather
+ * in the naive order, row after row (the contrast case for profiling: its
+ * re-reads mostly come from DRAM); with combo_segment_aggregate_rows: 3 nothing
+ * staged. */
 void combo_set_kernel_path(int path);
 
 /* Expert knob for the staged kernel, this thread only: tile width in elements

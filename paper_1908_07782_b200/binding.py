@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libcombo_b200.so")
 _lib = None
 
 COMBO_OK = 0
-PATH_AUTO, PATH_DIRECT, PATH_STAGED, PATH_TILE = 0, 1, 2, 5
+PATH_AUTO, PATH_DIRECT, PATH_STAGED, PATH_TILE, PATH_DIRECT_NAIVE = 0, 1, 2, 5, 6
 
 
 class ComboError(RuntimeError):

@@ -181,15 +181,16 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
 
     // candidate tiles: (T, box_w, nbx)
     struct Cand { int T, box_w, nbx; };
-    Cand cands[combo::kMaxBoxes + 2];
+    Cand cands[combo::kMaxBoxes + 3];
     int nc = 0;
     if (unaligned) {
         // every box carries 256 - V columns of the tile plus room for the row phase
         for (int n = 1; n <= combo::kMaxBoxes; ++n) cands[nc++] = {(256 - V) * n, 256, n};
     } else {
-        // with very many binary32 rows two stages of 256 columns do not fit: a half-width box
-        // (512 bytes per row, still a whole item per row) keeps such inputs on the staged path
-        if (EB == 4) cands[nc++] = {128, 128, 1};
+        // with very many rows two stages of 256 columns do not fit: narrower boxes (512 or 256
+        // bytes per row) keep such inputs on the staged path
+        if (EB == 4) cands[nc++] = {64, 64, 1};
+        cands[nc++] = {128, 128, 1};
         for (int n = 1; n <= combo::kMaxBoxes; ++n) cands[nc++] = {256 * n, 256, n};
     }
     auto stage_bytes = [&](const Cand& c) { return (long long)narr * c.nbx * p.N * c.box_w * EB; };
@@ -209,16 +210,19 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
         // draining the ring, which narrower stages do faster, and tiles are handed out
         // dynamically, which balances better with more of them.  (Measured on shapes from
         // 8 x 256 K to 16 x 1 M floats: the 32 KB choice was the best or within 1 % of it;
-        // 8 x 1 M: 14.4 us with 64 KB stages, 13.5 us with 32 KB.)
-        int wide = -1, mid = -1, narrowest = -1;
+        // 8 x 1 M: 14.4 us with 64 KB stages, 13.5 us with 32 KB.)  Boxes narrower than 256
+        // columns are the last resort: the widest of them that fits.
+        int wide = -1, mid = -1, narrowest = -1, narrow_box = -1;
         for (int i = 0; i < nc; ++i) {
             if (!feasible(cands[i])) continue;
+            if (cands[i].box_w < 256) { narrow_box = i; continue; }
             if (narrowest < 0) narrowest = i;
             if (stage_bytes(cands[i]) <= 64 * 1024) wide = i;
-            if (stage_bytes(cands[i]) <= 32 * 1024 && cands[i].box_w == 256) mid = i;   // half-width boxes: last resort only
+            if (stage_bytes(cands[i]) <= 32 * 1024) mid = i;
         }
         pick = wide >= 0 ? wide : narrowest;
         if (wide >= 0 && tiles(cands[wide]) < 32LL * dev.sms && mid >= 0) pick = mid;
+        if (pick < 0) pick = narrow_box;
         if (pick < 0) return plan;
     }
     const Cand c = cands[pick];
@@ -433,22 +437,31 @@ cudaError_t launch_tile(const AggParams& p, const combo::TileMaps& maps, const S
     return launch_tile_r<2, false>(p, maps, plan, st);
 }
 
-cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo& dev, cudaStream_t st) {
+cudaError_t launch_direct(const AggParams& p, int EB, bool sgd, const DeviceInfo& dev, cudaStream_t st,
+                          bool worker_major) {
     const int V = 16 / EB;
     const long long groups = (p.width + V - 1) / V + 1;
-    // x over the groups of a row, y = worker; about 32 resident CTAs per SM over all workers
-    long long bx = (groups + 255) / 256;
-    long long cap = ((long long)dev.sms * 32 + p.N - 1) / p.N;
-    if (cap < 1) cap = 1;
-    if (bx > cap) bx = cap;
-    const dim3 grid((unsigned)bx, (unsigned)p.N);
+    const long long blocks_per_row = (groups + 255) / 256;
+    const long long total = blocks_per_row * p.N;
+    // persistent CTAs, eight per SM, that take the blocks in their numbered order
+    const long long cap = (long long)dev.sms * 8;
+    const unsigned grid = (unsigned)(total < cap ? total : cap);
+    const int wm = worker_major ? 1 : 0;
+    const size_t smem = (size_t)(p.R + 1) * 16;          // providers and coefficients of two segments
+    cudaError_t e = cudaSuccess;
     if (EB == 4) {
-        if (sgd) combo::k_direct<4, true><<<grid, 256, 0, st>>>(p);
-        else combo::k_direct<4, false><<<grid, 256, 0, st>>>(p);
+        if (sgd) {
+            if (smem > 48 * 1024) e = cudaFuncSetAttribute(combo::k_direct<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e == cudaSuccess) combo::k_direct<4, true><<<grid, 256, smem, st>>>(p, blocks_per_row, wm);
+        } else {
+            if (smem > 48 * 1024) e = cudaFuncSetAttribute(combo::k_direct<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e == cudaSuccess) combo::k_direct<4, false><<<grid, 256, smem, st>>>(p, blocks_per_row, wm);
+        }
     } else {
-        combo::k_direct<2, false><<<grid, 256, 0, st>>>(p);
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(combo::k_direct<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) combo::k_direct<2, false><<<grid, 256, smem, st>>>(p, blocks_per_row, wm);
     }
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // widest column range one launch takes: a multiple of 64 elements (shards start on 16-byte
@@ -509,7 +522,7 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
     const bool sgd = grads != nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    bool want_staged = t_force_path != 1;
+    bool want_staged = t_force_path != 1 && t_force_path != 6;
     if (t_force_path == 0 && (long long)N * width < (1 << 16)) want_staged = false;   // too small to pipeline
     if (want_staged && t_force_path != 2) {
         // short inputs: one tile per CTA, several CTAs per SM
@@ -536,7 +549,7 @@ combo_status aggregate_cols(const void* in, const void* grads, float lr, void* o
             return COMBO_OK;
         }
     }
-    cudaError_t e = launch_direct(p, EB, sgd, *dev, st);
+    cudaError_t e = launch_direct(p, EB, sgd, *dev, st, t_force_path == 6);
     if (e != cudaSuccess) return cuda_fail(e, "direct aggregation launch");
     t_last_path = 1;
     return COMBO_OK;
@@ -1091,7 +1104,7 @@ combo_status combo_device_status(void) {
 
 int combo_last_kernel_path(void) { return t_last_path; }
 
-void combo_set_kernel_path(int path) { t_force_path = (path == 1 || path == 2 || path == 3 || path == 5) ? path : 0; }
+void combo_set_kernel_path(int path) { t_force_path = (path == 1 || path == 2 || path == 3 || path == 5 || path == 6) ? path : 0; }
 
 void combo_set_tuning(int tile_elems, int stages) {
     t_tile = tile_elems > 0 ? tile_elems : 0;

@@ -352,34 +352,102 @@ struct ProviderIter {
     }
 };
 
+// One output element straight from the definition (providers, weight sum and coefficients
+// worked out on the spot): for blocks that span more than two segments (segments shorter
+// than a block), where the per-block tables below do not reach.
 template <int EB, bool SGD>
-__global__ void __launch_bounds__(256) k_direct(const AggParams p) {
+__device__ __noinline__ void direct_element(const AggParams& p, int w, long long c) {
+    ProviderIter pi(p, w, (p.p_begin + c) / p.L);
+    float den = 0.0f;
+    bool first = true;
+    for (int k = pi.next(); k >= 0; k = pi.next()) {
+        const float D = p.weights ? p.weights[k] : 1.0f;
+        den = first ? D : __fadd_rn(den, D);
+        first = false;
+    }
+    pi.rewind();
+    float acc = 0.0f;
+    first = true;
+    for (int k = pi.next(); k >= 0; k = pi.next()) {
+        const float cf = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+        const float x = direct_x<EB, SGD>(p, k, c);
+        acc = first ? __fmul_rn(cf, x) : fmaf(cf, x, acc);
+        first = false;
+    }
+    ElemOps<EB>::store(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c) * EB, acc);
+}
+
+// Work is cut into blocks of 256 column groups of one worker's row.  The blocks are numbered
+// with the WORKER running fastest, and CTAs take them in that order: at any moment the
+// resident CTAs work on all workers' rows over the same narrow band of columns, so a provider
+// row's piece that one worker has brought into L2 is still there when the R other workers
+// that selected it ask for it -- the gather's re-reads are served by L2 and DRAM sees each
+// input element about once.  (worker_major = 1 numbers the blocks row after row instead: the
+// naive order, in which the re-reads of a row are spread over the whole run and mostly come
+// from DRAM; kept as the contrast case for profiling.)
+//
+// Per block the providers and coefficients of the (at most two) segments it touches are
+// worked out once, into shared memory: slot s of [2][R+1] holds the provider list and the
+// coefficients of segment la + s, la = the segment of the block's first column.
+template <int EB, bool SGD>
+__global__ void __launch_bounds__(256) k_direct(const AggParams p, long long blocks_per_row, int worker_major) {
     constexpr int V = ElemOps<EB>::V;
+    extern __shared__ __align__(16) unsigned char dsm[];
+    const int cap = p.R + 1;
+    int* s_prov = reinterpret_cast<int*>(dsm);                       // [2][cap]
+    float* s_coef = reinterpret_cast<float*>(s_prov + 2 * cap);      // [2][cap]
+    __shared__ int s_np[2];
+    __shared__ float s_den[2];
     const long long G = (p.width + V - 1) / V + 1;      // groups per row, phase spill included
     const bool rows_aligned = (p.pitch % V) == 0;
-    // grid: x strides over the groups of a row, y = worker
-    const int w = blockIdx.y;
-    const int a_w = (int)(((long long)w * p.pitch) & (V - 1));
-    for (long long g = blockIdx.x * 256LL + threadIdx.x; g < G; g += (long long)gridDim.x * 256LL) {
+    const long long total = blocks_per_row * p.N;
+    for (long long q = blockIdx.x; q < total; q += gridDim.x) {
+        const long long blk = worker_major ? q % blocks_per_row : q / p.N;
+        const int w = (int)(worker_major ? q / blocks_per_row : q % p.N);
+        const int a_w = (int)(((long long)w * p.pitch) & (V - 1));
+        // first column the block can touch and its segment
+        long long cfirst = blk * 256LL * V - a_w;
+        if (cfirst < 0) cfirst = 0;
+        if (cfirst >= p.width) continue;                                 // uniform: nothing in this block
+        const long long la = (p.p_begin + cfirst) / p.L;
+        __syncthreads();                                                 // the previous block's readers are done
+        if (threadIdx.x < 2) {
+            // the provider list in the fixed order and the sum of the weights in that order
+            const int sl = threadIdx.x;
+            int np = 0;
+            float den = 0.0f;
+            if (la + sl < p.S) {
+                ProviderIter pi(p, w, la + sl);
+                for (int k = pi.next(); k >= 0; k = pi.next()) {
+                    const float D = p.weights ? p.weights[k] : 1.0f;
+                    den = np == 0 ? D : __fadd_rn(den, D);
+                    s_prov[sl * cap + np++] = k;
+                }
+            }
+            s_np[sl] = np;
+            s_den[sl] = den;
+        }
+        __syncthreads();
+        for (int t = threadIdx.x; t < 2 * cap; t += 256) {
+            const int sl = t / cap, r = t - sl * cap;
+            if (r < s_np[sl]) s_coef[t] = __fdiv_rn(p.weights ? p.weights[s_prov[t]] : 1.0f, s_den[sl]);
+        }
+        __syncthreads();
+        const long long g = blk * 256LL + threadIdx.x;
+        if (g >= G) continue;
         const long long c0 = g * V - a_w;
         const long long lo = c0 < 0 ? 0 : c0;
         const long long hi = (c0 + V > p.width) ? p.width : c0 + V;
         if (lo >= hi) continue;
         const long long l_lo = (p.p_begin + lo) / p.L, l_hi = (p.p_begin + hi - 1) / p.L;
-        if (hi - lo == V && l_lo == l_hi && rows_aligned) {
-            ProviderIter pi(p, w, l_lo);
-            float den = 0.0f;
-            bool first = true;
-            for (int k = pi.next(); k >= 0; k = pi.next()) {
-                const float D = p.weights ? p.weights[k] : 1.0f;
-                den = first ? D : __fadd_rn(den, D);
-                first = false;
-            }
-            pi.rewind();
+        if (hi - lo == V && l_lo == l_hi && rows_aligned && l_lo - la < 2) {
+            const int sl = (int)(l_lo - la);
+            const int np = s_np[sl];
+            const int* prov = s_prov + sl * cap;
+            const float* coef = s_coef + sl * cap;
             float acc[V], x[V];
-            first = true;
-            for (int k = pi.next(); k >= 0; k = pi.next()) {
-                const size_t off = ((size_t)k * (size_t)p.pitch + (size_t)c0) * EB;
+            for (int r = 0; r < np; ++r) {
+                const size_t off = ((size_t)prov[r] * (size_t)p.pitch + (size_t)c0) * EB;
                 GroupLoad<EB, 16>::run(p.in + off, x);
                 if (SGD) {
                     float gx[V];
@@ -387,35 +455,28 @@ __global__ void __launch_bounds__(256) k_direct(const AggParams p) {
 #pragma unroll
                     for (int i = 0; i < V; ++i) x[i] = fmaf(-p.lr, gx[i], x[i]);
                 }
-                const float c = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
-                if (first) {
+                const float c = coef[r];
+                if (r == 0) {
 #pragma unroll
                     for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(c, x[i]);
                 } else {
 #pragma unroll
                     for (int i = 0; i < V; ++i) acc[i] = fmaf(c, x[i], acc[i]);
                 }
-                first = false;
             }
             ElemOps<EB>::store_vec(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c0) * EB, acc);
         } else {
             for (long long c = lo; c < hi; ++c) {
-                ProviderIter pi(p, w, (p.p_begin + c) / p.L);
-                float den = 0.0f;
-                bool first = true;
-                for (int k = pi.next(); k >= 0; k = pi.next()) {
-                    const float D = p.weights ? p.weights[k] : 1.0f;
-                    den = first ? D : __fadd_rn(den, D);
-                    first = false;
-                }
-                pi.rewind();
+                const long long sl64 = (p.p_begin + c) / p.L - la;
+                if (sl64 >= 2) { direct_element<EB, SGD>(p, w, c); continue; }
+                const int sl = (int)sl64;
+                const int np = s_np[sl];
+                const int* prov = s_prov + sl * cap;
+                const float* coef = s_coef + sl * cap;
                 float acc = 0.0f;
-                first = true;
-                for (int k = pi.next(); k >= 0; k = pi.next()) {
-                    const float cf = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
-                    const float x = direct_x<EB, SGD>(p, k, c);
-                    acc = first ? __fmul_rn(cf, x) : fmaf(cf, x, acc);
-                    first = false;
+                for (int r = 0; r < np; ++r) {
+                    const float x = direct_x<EB, SGD>(p, prov[r], c);
+                    acc = r == 0 ? __fmul_rn(coef[r], x) : fmaf(coef[r], x, acc);
                 }
                 ElemOps<EB>::store(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c) * EB, acc);
             }
@@ -794,6 +855,20 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
                 }
             }
         }
+    } else if (GB == 16 && interior && box_payload <= 256) {
+        // quarter-kilobyte row pieces (so many rows that wider ones do not fit): a warp takes
+        // two rows at a time, one per half-warp, each lane its 16 bytes
+        const int half = lane >> 4, hl = lane & 15;
+        RowCtx<RMAX> c;
+        const uint32_t lane_base = stage_s + hl * 16;
+        unsigned char* ocol = p.out + (size_t)t0 * EB + hl * 16;
+        for (int u = u_begin; u < u_end; u += 2) {
+            const int myrow = u + half;
+            if (myrow < u_end && hl * 16 < box_payload) {
+                load_entry<RMAX>(tab0 + (size_t)myrow * ENT, c);
+                item_fast<EB, GB, RMAX, (RT >= 0)>(lane_base, c, R, ocol + (size_t)myrow * pitch_bytes, 0xffu);
+            }
+        }
     } else if (interior) {
         // every unit is whole and lies in segment l0: the lean loop, rows outside, boxes inside
         RowCtx<RMAX> c;
@@ -826,7 +901,7 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
                 const int ib = xb * box_payload + ch * 512;          // byte offset of the item in the row
                 const uint32_t ubase = stage_s + xb * block_bytes + ch * 512 + lane * GB;
                 bool done = false;
-                if (GB == 16) {
+                if (GB == 16 && ch * 512 + lane * 16 < box_payload) {
                     const long long c0 = t0 + (ib + lane * 16) / EB;
                     const bool whole = c0 + V <= p.width;
                     const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
