@@ -23,6 +23,10 @@ thread_local int t_force_path = 0;
 thread_local int t_tile = 0;
 thread_local int t_stages = 0;
 thread_local int t_overlap = 1;
+#ifndef COMBO_DENSE_MAX
+#define COMBO_DENSE_MAX 32
+#endif
+constexpr int kDenseMaxWorkers = COMBO_DENSE_MAX;   // most workers the dense evaluation of many replicas is chosen for
 constexpr long long kTileMaxCtas = 1LL << 18;   // largest grid the one-tile-per-CTA kernel is chosen for
 
 struct DeviceInfo {
@@ -170,13 +174,28 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     // except on the rarely used granules
     plan.rt = (((p.R >= 1 && p.R <= 4) || p.R == 8) && (plan.gb == 16 || (EB == 2 && plan.gb == 4))) ? p.R : -1;
     if (p.R > combo::kGenericR) plan.rt = -2;                       // the wide unspecialised kernel
-    const int rmax = plan.rt >= 0 ? plan.rt : (plan.rt == -2 ? combo::kStagedMaxR : combo::kGenericR);
+    // Many replicas among few workers (Section 5.2 sweeps R to 16 with 30 workers): whole tiles
+    // are evaluated densely, a block of output rows against all N staged rows, which reads
+    // each staged piece once per block instead of once per provider.  Measured with 30 workers
+    // of 11.7 M floats, S = 10: 0.66 of the peak for every R from 9 to 16, against 0.64 / 0.59 /
+    // 0.53 at R = 9 / 12 / 16 in the warp-per-row form (bfloat16: 0.39 against 0.35 / 0.30 /
+    // 0.24); with 40 and 48 workers at R = 12 the warp-per-row form wins (0.50 / 0.55 against
+    // 0.46 / 0.45), hence the limit of 32.  Needs rows of one 16-byte phase and every row
+    // readable (no newcomer).
+    bool any_newcomer = false;
+    for (int i = 0; i < 256; ++i) any_newcomer |= p.newcomer.w[i] != 0;
+    const bool dense = plan.rt == -2 && plan.gb == 16 && !any_newcomer && p.N <= kDenseMaxWorkers;
+    if (dense) plan.rt = -3;
+    const int rmax = combo::rmax_of(plan.rt);
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
     // the coefficient table holds every segment when that is small (no rebuilds on the way,
     // which matters for short kernels), else two segments at a time
+    const int dense_br = EB == 4 ? 8 : 4;
+    const unsigned dslot = dense ? round_up((unsigned)((p.N + dense_br - 1) / dense_br * (p.N + 1) * dense_br * 4), 128) : 0;
     const unsigned entry = (unsigned)combo::table_entry_bytes(rmax);
-    int tab_slots = ((unsigned long long)p.S * p.N * entry <= 24u * 1024u && p.S >= 2) ? p.S : 2;
-    unsigned table = round_up((unsigned)tab_slots * p.N * entry, 128);
+    const unsigned long long slot_bytes = (unsigned long long)p.N * entry + dslot;
+    int tab_slots = ((unsigned long long)p.S * slot_bytes <= 24u * 1024u && p.S >= 2) ? p.S : 2;
+    unsigned table = round_up((unsigned)tab_slots * p.N * entry, 128) + (unsigned)tab_slots * dslot;
     const long long budget = (long long)dev.smem_optin - header - table - 256;
 
     // candidate tiles: (T, box_w, nbx)
@@ -226,6 +245,7 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
         if (pick < 0) return plan;
     }
     const Cand c = cands[pick];
+    if (plan.rt == -3 && c.box_w != 256) plan.rt = -2;   // the dense form walks whole 512-byte chunks of 256-column boxes
     // Measured on B200: throughput peaks with about 96-128 KB of loads in flight per SM and
     // drops by 5-10 % beyond that, so the ring is kept that short (at least two stages; stages of
     // at most 32 KB, which fill and drain more often, may hold up to 160 KB together).
@@ -240,8 +260,9 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     // costs two consumer barriers and a round trip to the peer table: it shows in kernels of
     // a hundred microseconds with many segments)
     if (tab_slots < p.S) {
-        const unsigned long long whole = round_up((unsigned)((unsigned long long)p.S * p.N * entry), 128);
-        if ((unsigned long long)p.S * p.N * entry < (1u << 20) &&
+        const unsigned long long whole = round_up((unsigned)((unsigned long long)p.S * p.N * entry), 128) +
+                                         (unsigned long long)p.S * dslot;
+        if ((unsigned long long)p.S * slot_bytes < (1u << 20) &&
             (long long)(whole - table) <= budget - (long long)stages * stage_bytes(c)) {
             tab_slots = p.S;
             table = (unsigned)whole;
@@ -256,6 +277,8 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     p.stage_bytes = (unsigned)stage_bytes(c);
     p.tab_off = header;
     p.tab_slots = tab_slots;
+    p.dtab_off = header + round_up((unsigned)tab_slots * p.N * entry, 128);
+    p.dslot_bytes = (int)dslot;
     p.stage_off = header + table;
     p.n_tiles = tiles(c);
     for (int a = 0; a < narr; ++a)
@@ -303,6 +326,7 @@ cudaError_t launch_staged_r(const AggParams& p, const combo::TileMaps& maps, con
         case 4: return launch_staged_inst<EB, GB, SGD, 4>(p, maps, plan, st);
         case 8: return launch_staged_inst<EB, GB, SGD, 8>(p, maps, plan, st);
         case -2: return launch_staged_inst<EB, GB, SGD, -2>(p, maps, plan, st);
+        case -3: return launch_staged_inst<EB, GB, SGD, -3>(p, maps, plan, st);
         default: return launch_staged_inst<EB, GB, SGD, -1>(p, maps, plan, st);
     }
 }
@@ -343,7 +367,7 @@ StagedPlan plan_tile(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, cons
     if ((unsigned long long)p.width + 256 >= (1ull << 31)) return plan;   // TMA coordinates are signed 32-bit
     plan.rt = ((p.R >= 1 && p.R <= 4) || p.R == 8) ? p.R : -1;
     if (p.R > combo::kGenericR) plan.rt = -2;
-    const int rmax = plan.rt >= 0 ? plan.rt : (plan.rt == -2 ? combo::kStagedMaxR : combo::kGenericR);
+    const int rmax = combo::rmax_of(plan.rt);
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
     const unsigned table = round_up(2u * p.N * (unsigned)combo::table_entry_bytes(rmax), 128);
     // Tile: at least 1 KB of every row (256 binary32 or 512 bfloat16 columns; shorter row
@@ -853,7 +877,7 @@ combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, 
         long long d_max = (long long)n_local * (1 + 2 * R);
         if (d_max > N) d_max = N;
         const int rt = ((R >= 1 && R <= 4) || R == 8) ? R : (R > combo::kGenericR ? -2 : -1);
-        const int rmax = rt >= 0 ? rt : (rt == -2 ? combo::kStagedMaxR : combo::kGenericR);
+        const int rmax = combo::rmax_of(rt);
         combo::PullStagedParams q;
         memset(&q, 0, sizeof(q));
         q.ptr_off = 0;

@@ -45,6 +45,9 @@ constexpr int kStagedThreads = 32 + kConsumerThreads;
 constexpr int kMaxStages = 8;
 constexpr int kStagedMaxR = 16;            // most replicas the staged kernel takes (Section 5.2 sweeps R up to 16)
 constexpr int kGenericR = 8;               // replicas of the unspecialised kernel; beyond: the wide one
+// Replicas a kernel instance is built for: RT >= 0 exactly RT; -1 any up to kGenericR; -2 any up
+// to kStagedMaxR; -3 the same with the dense evaluation of whole tiles (see aggregate_dense).
+__host__ __device__ constexpr int rmax_of(int rt) { return rt >= 0 ? rt : (rt == -1 ? 8 : 16); }
 constexpr int kMaxClasses = 8;
 constexpr int kMaxBoxes = 8;              // x-boxes per tile
 constexpr uint32_t kWaitCap = 1u << 23;   // polls before a wait is declared dead
@@ -93,6 +96,8 @@ struct AggParams {
     int row_bytes;       // shared-memory bytes per staged row of one box = box_w * e
     unsigned tab_off;    // byte offset of the coefficient table in shared memory
     int tab_slots;       // segments the table holds: all S of them, or 2 (rebuilt on the way)
+    unsigned dtab_off;   // byte offset of the dense coefficient blocks (dense mode only)
+    int dslot_bytes;     // bytes of one segment's dense blocks
     unsigned stage_off;  // byte offset of stage 0
     unsigned stage_bytes;
     TileSlot* sched;     // tile dispenser of this launch
@@ -167,8 +172,13 @@ __device__ __forceinline__ f32x2 mul2(f32x2 c, f32x2 x) {
     return d;
 }
 __device__ __forceinline__ f32x2 fma2(f32x2 c, f32x2 x, f32x2 acc) {
+#ifdef COMBO_SCALAR_FMA
+    return pair_bits(__float_as_uint(fmaf(pair_lo(c), pair_lo(x), pair_lo(acc))),
+                     __float_as_uint(fmaf(pair_hi(c), pair_hi(x), pair_hi(acc))));
+#else
     asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(c), "l"(x));
     return acc;
+#endif
 }
 // a 32-bit word holding two bf16 -> the pair of their binary32 values
 __device__ __forceinline__ f32x2 bf16x2_widen(uint32_t w) { return pair_bits(w << 16, w & 0xffff0000u); }
@@ -762,10 +772,11 @@ struct WarpShare {
     static constexpr int PIECES = 16 / GB;                // pieces a lane owns per item
     static constexpr int PSTRIDE = 32 * GB;               // bytes between a lane's pieces
     int u_begin, u_end, row_begin, xb_begin;
+    int cw, nwarps;                                       // this warp's number among those sharing the tile
     int box_payload;                                      // tile bytes per row held by one x-box
     size_t pitch_bytes;
     unsigned pmask[CPB];    // store masks of the unit's chunks: bit i = piece i of this lane lies inside the payload
-    __device__ __forceinline__ WarpShare(const AggParams& p, int cw, int nwarps, int lane) {
+    __device__ __forceinline__ WarpShare(const AggParams& p, int cw_, int nwarps_, int lane) : cw(cw_), nwarps(nwarps_) {
         box_payload = (p.T / p.nbx) * EB;
         const int n_units = p.N * p.nbx;
         const int upw = (n_units + nwarps - 1) / nwarps;
@@ -784,6 +795,139 @@ struct WarpShare {
     }
 };
 
+// ---------------------------------------------------------------- dense evaluation (many replicas)
+// With R + 1 providers per output the warp-per-row loop reads R + 1 staged rows per output
+// row; beyond R of about 8 those shared-memory reads, not HBM, set the pace.  When R + 1 is a
+// good part of N (the paper sweeps R up to 16 with 30 workers, Section 5.2) it is cheaper to
+// take a BLOCK of BR output rows at once and walk over ALL N staged rows: each staged piece
+// is read once per block and multiplied into the BR accumulators with that row's
+// coefficients, which are zero where the row is not a provider.  fma(0, x, acc) leaves acc
+// as it is for finite x, so every output still sees exactly the fixed order of Eq. 3 (own
+// term first, then providers ascending).  Rows must hold finite values, all of them, since
+// every row meets every accumulator; not used when a newcomer flag is set (a newcomer's own
+// row must never be read).
+// A block is as many output rows as keep the accumulators within 32 registers of pairs: 8 of
+// binary32 (a lane's 16 bytes are 4 elements), 4 of bfloat16 (8 elements).  Per staged row a
+// unit then reads 512 bytes of data and 32 or 16 bytes of coefficients.  (Twice the columns
+// per lane would halve the coefficient reads per output but spills registers, which measured
+// no faster than the warp-per-row form.)
+template <int EB> struct DenseRows {
+    static constexpr int BR = (EB == 4) ? 8 : 4;
+    static constexpr int CH = 1;                     // 512-byte chunks a unit spans
+};
+
+// Dense coefficient blocks of `nslots` segments: [slot][block][k = 0..N][BR] floats; k < N:
+// coefficient of staged row k for output row BR*block + b, zero if it is not a provider or is
+// the output row itself; k = N: the output row's own coefficient.
+template <int EB>
+__device__ __forceinline__ void build_dense_table(const AggParams& p, unsigned char* dtab, int R, int l0_build,
+                                                  int nslots, int t, int nthreads) {
+    constexpr int BR = DenseRows<EB>::BR;
+    const int N = p.N;
+    const int nblk = (N + BR - 1) / BR;
+    for (int q = t; q < nslots * nblk * BR; q += nthreads) {
+        const int slot = q / (nblk * BR), w = q - slot * nblk * BR;     // w may be a padding row >= N
+        const int l = l0_build + slot;
+        if (l >= p.S) continue;
+        float* col = reinterpret_cast<float*>(dtab + (size_t)slot * p.dslot_bytes) +
+                     (size_t)(w / BR) * (N + 1) * BR + (w % BR);
+        for (int k = 0; k <= N; ++k) col[(size_t)k * BR] = 0.0f;
+        if (w >= N) continue;
+        const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
+        float den = p.weights ? p.weights[w] : 1.0f;
+        for (int r = 0; r < R; ++r)
+            if (peers[r] >= 0) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+        col[(size_t)N * BR] = __fdiv_rn(p.weights ? p.weights[w] : 1.0f, den);
+        for (int r = 0; r < R; ++r) {
+            const int k = peers[r];
+            if (k >= 0) col[(size_t)k * BR] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+        }
+    }
+}
+
+// the BR coefficients of one staged row, each duplicated into a pair
+template <int BR>
+__device__ __forceinline__ void dense_coefs(uint32_t a, f32x2 (&c)[BR]) {
+#pragma unroll
+    for (int b = 0; b < BR; b += 4) {
+        const uint4 v = lds128(a + b * 4);
+        c[b] = pair_bits(v.x, v.x); c[b + 1] = pair_bits(v.y, v.y);
+        c[b + 2] = pair_bits(v.z, v.z); c[b + 3] = pair_bits(v.w, v.w);
+    }
+}
+
+// A whole tile lying in one segment, dense: warp number cw of nwarps takes the units
+// (row block, group of CH chunks) cw, cw + nwarps, ...
+template <int EB>
+__device__ __forceinline__ void aggregate_dense(const AggParams& p, uint32_t stage_s, const unsigned char* dtab0,
+                                                long long t0, int cw, int nwarps, int lane) {
+    constexpr int BR = DenseRows<EB>::BR;
+    constexpr int CH = DenseRows<EB>::CH;
+    constexpr int NP = ElemOps<EB>::V / 2;          // pairs per 16-byte piece
+    const int N = p.N;
+    const int nblk = (N + BR - 1) / BR;
+    const int box_payload = (p.T / p.nbx) * EB;     // a multiple of CH * 512 (checked by the planner)
+    const int groups_per_box = box_payload / (CH * 512);
+    const int groups = p.nbx * groups_per_box;
+    const int block_bytes = N * p.row_bytes;
+    const size_t pitch_bytes = (size_t)p.pitch * EB;
+    const uint32_t dt_s = smem_u32(dtab0);
+    for (int u = cw; u < nblk * groups; u += nwarps) {
+        const int blk = u / groups, gq = u - blk * groups;
+        const int xb = gq / groups_per_box, gi = gq - xb * groups_per_box;
+        const int w0 = blk * BR;
+        const int col_off = gi * CH * 512 + lane * 16;                 // byte offset inside the box payload
+        const uint32_t base = stage_s + xb * block_bytes + col_off;
+        uint32_t ct = dt_s + (uint32_t)(blk * (N + 1) * BR * 4);
+        f32x2 acc[BR][CH * NP], x[CH * NP], c[BR];
+        // own terms first
+        dense_coefs<BR>(ct + (uint32_t)(N * BR * 4), c);
+#pragma unroll
+        for (int b = 0; b < BR; ++b) {
+            const int w = w0 + b < N ? w0 + b : N - 1;                  // padding rows: any staged row, coefficient 0
+#pragma unroll
+            for (int h = 0; h < CH; ++h) {
+                f32x2 xx[NP];
+                PairLoad<EB, 16>::run(base + w * p.row_bytes + h * 512, xx);
+#pragma unroll
+                for (int i = 0; i < NP; ++i) acc[b][h * NP + i] = mul2(c[b], xx[i]);
+            }
+        }
+        // then every staged row in ascending order
+        uint32_t xa = base;
+#pragma unroll 1
+        for (int k = 0; k < N; ++k) {
+#pragma unroll
+            for (int h = 0; h < CH; ++h) {
+                f32x2 xx[NP];
+                PairLoad<EB, 16>::run(xa + h * 512, xx);
+#pragma unroll
+                for (int i = 0; i < NP; ++i) x[h * NP + i] = xx[i];
+            }
+            dense_coefs<BR>(ct, c);
+#pragma unroll
+            for (int b = 0; b < BR; ++b)
+#pragma unroll
+                for (int i = 0; i < CH * NP; ++i) acc[b][i] = fma2(c[b], x[i], acc[b][i]);
+            xa += p.row_bytes;
+            ct += BR * 4;
+        }
+        unsigned char* o = p.out + (size_t)w0 * pitch_bytes + (size_t)t0 * EB + (size_t)xb * box_payload + col_off;
+#pragma unroll
+        for (int b = 0; b < BR; ++b) {
+            if (w0 + b < N) {
+#pragma unroll
+                for (int h = 0; h < CH; ++h) {
+                    f32x2 r[NP];
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) r[i] = acc[b][h * NP + i];
+                    PairStore<EB, 16>::run(o + (size_t)b * pitch_bytes + h * 512, r, 0xffu);
+                }
+            }
+        }
+    }
+}
+
 // One warp's share of a staged tile: Eq. 3 in the fixed order for every unit of `ws`, results
 // stored to the output rows.  `stage` holds the tile (its shared-window address is stage_s),
 // tab0 the table entries of segment l0 (those of l0 + 1 follow them), m_bnd is the local
@@ -792,9 +936,9 @@ template <int EB, int GB, int RT>
 __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpShare<EB, GB>& ws,
                                                const unsigned char* stage, uint32_t stage_s,
                                                const unsigned char* tab0, long long tile, long long m_bnd,
-                                               int lane) {
+                                               int lane, const unsigned char* dtab0 = nullptr) {
     constexpr int V = ElemOps<EB>::V;
-    constexpr int RMAX = (RT >= 0) ? RT : (RT == -2 ? kStagedMaxR : kGenericR);
+    constexpr int RMAX = rmax_of(RT);
     constexpr int ENT = table_entry_bytes(RMAX);
     constexpr int CPB = WarpShare<EB, GB>::CPB;
     constexpr int PIECES = WarpShare<EB, GB>::PIECES;
@@ -808,6 +952,12 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
     const long long t0 = tile * (long long)p.T;
     const long long t1 = (t0 + p.T < p.width) ? t0 + p.T : p.width;
     const bool interior = (m_bnd >= t1) && (t0 + p.T <= p.width);   // one segment, whole tile
+    if constexpr (RT == -3 && GB == 16) {
+        if (interior) {
+            aggregate_dense<EB>(p, stage_s, dtab0, t0, ws.cw, ws.nwarps, lane);
+            return;
+        }
+    }
 
     int row = ws.row_begin, xb = ws.xb_begin;
     if (GB < 16 && interior) {
@@ -944,7 +1094,7 @@ __global__ void __launch_bounds__(kStagedThreads, 1)
 k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     // RT: the number of replicas the kernel is specialised on, -1 = any up to kGenericR,
     // -2 = any up to kStagedMaxR
-    constexpr int RMAX = (RT >= 0) ? RT : (RT == -2 ? kStagedMaxR : kGenericR);
+    constexpr int RMAX = rmax_of(RT);
     constexpr int ENT = table_entry_bytes(RMAX);
     extern __shared__ __align__(128) unsigned char smem[];
     StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
@@ -1101,12 +1251,16 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
 
     // The first tile's table does not depend on the staged data: build it while the
     // first TMA loads are in flight.
+    constexpr bool DENSE = (RT == -3 && GB == 16);
+    unsigned char* dtab = smem + p.dtab_off;               // dense coefficient blocks, one set per table slot
     if ((long long)blockIdx.x < p.n_tiles) {
         if (whole_table) {
             build_coef_table<EB, RMAX>(p, tab, R, 0, p.S, ctid, kConsumerThreads);
+            if (DENSE) build_dense_table<EB>(p, dtab, R, 0, p.S, ctid, kConsumerThreads);
         } else {
             cached_l0 = (int)((p.p_begin + (long long)blockIdx.x * p.T) / p.L);
             build_coef_table<EB, RMAX>(p, tab, R, cached_l0, 2, ctid, kConsumerThreads);
+            if (DENSE) build_dense_table<EB>(p, dtab, R, cached_l0, 2, ctid, kConsumerThreads);
         }
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(7); return; }
     }
@@ -1129,6 +1283,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             // table for segments l0 and l0+1 (rebuilt at most S times per CTA)
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(4); return; }
             build_coef_table<EB, RMAX>(p, tab, R, m_l0, 2, ctid, kConsumerThreads);
+            if (DENSE) build_dense_table<EB>(p, dtab, R, m_l0, 2, ctid, kConsumerThreads);
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
             cached_l0 = m_l0;
         }
@@ -1139,7 +1294,8 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(6); return; }
         }
 
-        aggregate_tile<EB, GB, RT>(p, ws, stage, stage_s, tab0, tile, m_bnd, lane);
+        aggregate_tile<EB, GB, RT>(p, ws, stage, stage_s, tab0, tile, m_bnd, lane,
+                                   DENSE ? dtab + (size_t)(whole_table ? m_l0 : 0) * p.dslot_bytes : nullptr);
 
         // The fused step rewrote the stage with ordinary stores; the copy that refills it goes
         // through the asynchronous proxy, so the two are ordered by a proxy fence.
@@ -1162,7 +1318,7 @@ constexpr int kTileThreads = 32 * kTileWarps;
 template <int EB, int GB, bool SGD, int RT>
 __global__ void __launch_bounds__(kTileThreads)
 k_tile(const AggParams p, const __grid_constant__ TileMaps maps) {
-    constexpr int RMAX = (RT >= 0) ? RT : (RT == -2 ? kStagedMaxR : kGenericR);
+    constexpr int RMAX = rmax_of(RT);
     extern __shared__ __align__(128) unsigned char smem[];
     StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

@@ -34,7 +34,8 @@ def test_select_peers_online_bit_exact(N, S, R):
 
 
 CASES = [(8, 40_000, 4, 2, torch.float32), (13, 50_001, 5, 4, torch.float32), (32, 20_004, 8, 3, torch.float32),
-         (128, 5_002, 16, 4, torch.bfloat16), (20, 30_000, 3, 6, torch.bfloat16), (6, 3_000, 2, 3, torch.float32)]
+         (128, 5_002, 16, 4, torch.bfloat16), (20, 30_000, 3, 6, torch.bfloat16), (6, 3_000, 2, 3, torch.float32),
+         (24, 40_000, 4, 10, torch.float32), (30, 24_000, 5, 12, torch.bfloat16)]    # many replicas
 
 
 @pytest.mark.parametrize("N,P,S,R,dtype", CASES)
@@ -83,4 +84,40 @@ def test_aggregate_members(N, P, S, R, dtype, path):
     # offline workers keep their model bit for bit
     for v in np.flatnonzero(active == 0):
         assert (got[v] == xb[v]).all()
+    combo.combo_device_status()
+
+
+@pytest.mark.parametrize("N,P,S,R,dtype", [(24, 60_000, 4, 10, torch.float32), (30, 48_000, 5, 14, torch.bfloat16),
+                                           (21, 60_004, 3, 9, torch.float32)])
+def test_many_replicas_with_absent_peers_and_no_newcomer(N, P, S, R, dtype):
+    # offline workers and pulls that found no peer, but nobody new: with R > 8 among few workers
+    # whole tiles are evaluated densely (every staged row meets every output with a coefficient
+    # that is zero for non-providers); the bits must still be those of the fixed order
+    rng = np.random.default_rng(N + R)
+    g = torch.Generator().manual_seed(N)
+    x = (torch.randn(N, P, generator=g) * 0.05 + 0.01).to(dtype)
+    w = torch.randint(500, 1501, (N,), generator=g).float()
+    active = np.ones(N, np.uint8)
+    active[rng.choice(N, size=3, replace=False)] = 0
+    idx_np = oracle.select_peers_active(6, 2, N, S, R, active)
+    online = np.flatnonzero(active)
+    idx_np[online[0], 0, :] = -1                       # a segment with no peer at all
+    idx_np[online[1], S - 1, R // 2:] = -1             # half the pulls missing
+    xb = to_bits(x)
+    ordered = oracle.segment_aggregate_members(xb, idx_np, S, R, w.numpy(), np.zeros(N, np.uint8), ordered=True)
+    xd = x.to(DEV)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    outs = []
+    for path in (combo.PATH_STAGED, combo.PATH_DIRECT):
+        out = torch.empty_like(xd)
+        combo.combo_set_kernel_path(path)
+        try:
+            combo.combo_segment_aggregate_members(xd, out, w.to(DEV), idx, None, N, P, S, R)
+            torch.cuda.synchronize()
+            assert combo.combo_last_kernel_path() == path
+        finally:
+            combo.combo_set_kernel_path(combo.PATH_AUTO)
+        assert (to_bits(out).view(np.uint8) == ordered.view(np.uint8)).all(), path
+        outs.append(out)
+    assert torch.equal(outs[0], outs[1])
     combo.combo_device_status()

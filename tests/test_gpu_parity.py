@@ -117,6 +117,11 @@ MEDIUM = [
     (230, 3_004, 2, 4, torch.float32, True),
     (250, 4_000, 3, 2, torch.bfloat16, False),    # the same in bf16 (128-column boxes)
     (140, 6_000, 3, 3, torch.float32, True),      # 512-byte row pieces
+    (30, 40_000, 10, 12, torch.float32, True),    # many replicas among few workers: dense evaluation of whole tiles
+    (30, 40_000, 10, 16, torch.bfloat16, False),
+    (33, 20_000, 3, 9, torch.float32, False),     # a last block of one row
+    (32, 20_000, 4, 13, torch.bfloat16, True),
+    (34, 20_000, 4, 13, torch.float32, True),     # too many workers for it: the warp-per-row form
 ]
 
 
