@@ -221,12 +221,17 @@ int oracle_segment_aggregate(const void *in, const void *grads, double lr, int e
 }
 
 /* ------------------------------------------------------------------ */
-/* The same round in binary32 with one fixed operation order: provider */
-/* order is self first, then peers ascending; the weights are          */
-/* normalised first (c_j = |D_j| / sum, one IEEE division per          */
-/* provider), then out = c_self*x_self, out = fma(c_j, x_j, out).      */
-/* The local step is x = fma(-lr, g, x) rounded to binary32.  A bf16   */
-/* result is the binary32 result rounded to nearest even.  This is a   */
+/* The same round in binary32 with one fixed operation order, Eq. 3 as */
+/* it is written: provider order is self first, then peers ascending;  */
+/*   num = |D_self|*x_self, num = fma(|D_j|, x_j, num)                 */
+/*   den = |D_self|, den = den + |D_j|            (the same order)     */
+/*   out = num * (1/den)      (the reciprocal rounded to binary32)     */
+/* With a single provider the quotient is that provider's value and is */
+/* taken as such (out = x: R = 0 is the identity, bit for bit).  With  */
+/* weights == NULL every |D_j| is 1, the products are exact and num is */
+/* the plain sum in that order.  The local step is x = fma(-lr, g, x)  */
+/* rounded to binary32.  A bf16 result is the binary32 result rounded  */
+/* to nearest even.  This is a                                         */
 /* second, tighter yardstick for a binary32 implementation that uses   */
 /* the same order; it is itself pinned against the binary64 form.      */
 /* out: [N][p_end-p_begin] of float (elem 4) or uint16 bf16 (elem 2).  */
@@ -241,7 +246,6 @@ int oracle_segment_aggregate_ordered_f32(const void *in, const void *grads, floa
     if (grads && elem != 4) return 1;
     int64_t L = oracle_segment_length(P, S);
     int64_t width = p_end - p_begin;
-    float *coef = (float *)malloc(sizeof(float) * (size_t)(R + 1));
     for (int w = 0; w < N; ++w) {
         for (int l = 0; l < S; ++l) {
             int64_t a = (int64_t)l * L, b = a + L;
@@ -251,8 +255,7 @@ int oracle_segment_aggregate_ordered_f32(const void *in, const void *grads, floa
             const int32_t *peers = idx ? idx + ((size_t)w * S + l) * R : NULL;
             volatile float den = weights ? weights[w] : 1.0f;
             for (int r = 0; r < R; ++r) den = den + (weights ? weights[peers[r]] : 1.0f);
-            coef[0] = (weights ? weights[w] : 1.0f) / den;
-            for (int r = 0; r < R; ++r) coef[r + 1] = (weights ? weights[peers[r]] : 1.0f) / den;
+            volatile float rden = 1.0f / den;
             for (int64_t p = a; p < b; ++p) {
                 float acc = 0.0f;
                 for (int m = -1; m < R; ++m) {
@@ -261,16 +264,17 @@ int oracle_segment_aggregate_ordered_f32(const void *in, const void *grads, floa
                     float x = (elem == 4) ? ((const float *)in)[off]
                                           : bf16_to_f32(((const uint16_t *)in)[off]);
                     if (grads) x = fmaf(-lr, ((const float *)grads)[off], x);
-                    if (m < 0) { volatile float prod = coef[0] * x; acc = prod; }
-                    else acc = fmaf(coef[m + 1], x, acc);
+                    float D = weights ? weights[j] : 1.0f;
+                    if (m < 0) { volatile float prod = D * x; acc = (R == 0) ? x : prod; }
+                    else acc = fmaf(D, x, acc);
                 }
+                if (R > 0) { volatile float q = acc * rden; acc = q; }
                 size_t o = (size_t)w * (size_t)width + (size_t)(p - p_begin);
                 if (elem == 4) ((float *)out)[o] = acc;
                 else ((uint16_t *)out)[o] = oracle_f32_to_bf16_rne(acc);
             }
         }
     }
-    free(coef);
     return 0;
 }
 
@@ -389,7 +393,6 @@ int oracle_segment_aggregate_members(const void *in, int elem, const float *weig
     if (N < 1 || P < 1 || S < 1 || R < 0 || (elem != 4 && elem != 2)) return 1;
     int64_t L = oracle_segment_length(P, S);
     int *prov = (int *)malloc(sizeof(int) * (size_t)(R + 1));
-    float *coef = (float *)malloc(sizeof(float) * (size_t)(R + 1));
     for (int w = 0; w < N; ++w) {
         for (int l = 0; l < S; ++l) {
             int64_t a = (int64_t)l * L, b = a + L;
@@ -402,13 +405,14 @@ int oracle_segment_aggregate_members(const void *in, int elem, const float *weig
                 if (k >= 0) prov[np++] = k;
             }
             if (np == 0) prov[np++] = w;
+            volatile float rden32 = 1.0f;
             if (mode == 1) {
                 volatile float den = 0.0f;
                 for (int q = 0; q < np; ++q) {
                     float D = weights ? weights[prov[q]] : 1.0f;
                     den = (q == 0) ? D : den + D;
                 }
-                for (int q = 0; q < np; ++q) coef[q] = (weights ? weights[prov[q]] : 1.0f) / den;
+                rden32 = 1.0f / den;
             }
             for (int64_t p = a; p < b; ++p) {
                 size_t o = (size_t)w * (size_t)P + (size_t)p;
@@ -421,19 +425,22 @@ int oracle_segment_aggregate_members(const void *in, int elem, const float *weig
                     }
                     ((double *)out)[o] = num / den;
                 } else {
+                    /* the fixed-order binary32 form, as in oracle_segment_aggregate_ordered_f32 */
                     float acc = 0.0f;
                     for (int q = 0; q < np; ++q) {
                         size_t off = (size_t)prov[q] * (size_t)P + (size_t)p;
                         float x = (elem == 4) ? ((const float *)in)[off] : bf16_to_f32(((const uint16_t *)in)[off]);
-                        if (q == 0) { volatile float prod = coef[0] * x; acc = prod; }
-                        else acc = fmaf(coef[q], x, acc);
+                        float D = weights ? weights[prov[q]] : 1.0f;
+                        if (q == 0) { volatile float prod = D * x; acc = (np == 1) ? x : prod; }
+                        else acc = fmaf(D, x, acc);
                     }
+                    if (np > 1) { volatile float qq = acc * rden32; acc = qq; }
                     if (elem == 4) ((float *)out)[o] = acc;
                     else ((uint16_t *)out)[o] = oracle_f32_to_bf16_rne(acc);
                 }
             }
         }
     }
-    free(prov); free(coef);
+    free(prov);
     return 0;
 }

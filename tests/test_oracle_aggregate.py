@@ -286,3 +286,26 @@ def test_bf16_storage_matches_exact_within_one_ulp():
     got = oracle.segment_aggregate_ordered_f32(bits, idx, S, R)
     ulp = 2.0 ** (np.floor(np.log2(np.abs(exact) + 1e-300)) - 7)
     assert (np.abs(bf16_to_f64(got) - exact) <= 0.5 * ulp * (1 + 1e-3)).all()
+
+
+def test_ordered_f32_is_eq3_as_written():
+    # Eq. 3 in binary32, in the fixed order: num = D_self*x_self, num = fma(D_j, x_j, num),
+    # den summed in the same order, out = num * (1/den).  With unit weights the products are
+    # exact, so num is the plain sequential sum, which numpy's binary32 adds reproduce.
+    rng = np.random.default_rng(21)
+    N, P, S, R = 7, 41, 3, 4
+    x = rng.normal(0, 0.05, (N, P)).astype(np.float32)
+    idx = oracle.select_peers(4, 2, N, S, R)
+    got = oracle.segment_aggregate_ordered_f32(x, idx, S, R)
+    L = -(-P // S)
+    rcp = np.float32(1.0) / np.float32(R + 1)
+    for i in range(N):
+        for p in range(P):
+            acc = x[i, p]
+            for k in idx[i, p // L]:
+                acc = np.float32(acc + x[k, p])
+            assert got[i, p] == np.float32(acc * rcp)
+    # unit weights given explicitly are the same computation, bit for bit
+    ones = np.ones(N, np.float32)
+    assert (oracle.segment_aggregate_ordered_f32(x, idx, S, R, weights=ones).view(np.uint32)
+            == got.view(np.uint32)).all()
