@@ -102,9 +102,15 @@ combo_status combo_select_peers_async(uint64_t seed, uint32_t round, int N, int 
  * they hold after the local update, Section 4.1 steps 3 and 4), so params_out
  * must not overlap params_in.
  *
- * Arithmetic: binary32.  den = |D_w| + |D_k1| + ... (peers ascending),
- * c_j = |D_j| / den (IEEE division), out = c_w*x_w, then out = fma(c_k, x_k, out)
- * for the peers in ascending order.  No fast-math, denormals kept.
+ * Arithmetic: binary32, Eq. 3 as it is written.  num = |D_w|*x_w, then
+ * num = fma(|D_k|, x_k, num) for the peers in ascending order;
+ * den = |D_w| + |D_k1| + ... in the same order; out = num * (1/den), the
+ * reciprocal rounded to binary32 (one IEEE division per worker and segment).
+ * A single provider is taken as it is (out = x).  With weights == NULL every
+ * |D_j| is 1: the products are exact and num is the plain sum in that order
+ * (bfloat16 rows are then added by the mixed-precision instruction
+ * add.rn.f32.bf16, which widens exactly and rounds once: the same bits).
+ * |D_j|*x must stay within the binary32 range.  No fast-math, denormals kept.
  *
  * params_in, params_out: float [N][P], base addresses 16-byte aligned.
  * weights: float[N] or NULL.  idx: int32[N][S][R], trusted (see

@@ -111,6 +111,7 @@ struct StagedPlan {
     int rt;          // R the kernel is specialised on, or -1
     size_t smem;
     int grid;
+    bool unw;        // bfloat16 rows with unit weights: the mixed-precision sum (see RowCtxU)
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -159,7 +160,7 @@ bool encode_class_map(CUtensorMap* map, const unsigned char* base, int EB, int j
 }
 
 StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, const DeviceInfo& dev) {
-    StagedPlan plan = {false, 16, -1, 0, 0};
+    StagedPlan plan = {false, 16, -1, 0, 0, false};
     const int V = 16 / EB;
     const int narr = sgd ? 2 : 1;
     if (p.R > combo::kStagedMaxR) return plan;
@@ -187,12 +188,13 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     const bool dense = plan.rt == -2 && plan.gb == 16 && !any_newcomer && p.N <= kDenseMaxWorkers;
     if (dense) plan.rt = -3;
     const int rmax = combo::rmax_of(plan.rt);
+    plan.unw = EB == 2 && !p.weights && !sgd && !dense && plan.gb != 2;
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
     // the coefficient table holds every segment when that is small (no rebuilds on the way,
     // which matters for short kernels), else two segments at a time
     const int dense_br = EB == 4 ? 8 : 4;
-    const unsigned dslot = dense ? round_up((unsigned)((p.N + dense_br - 1) / dense_br * (p.N + 1) * dense_br * 4), 128) : 0;
-    const unsigned entry = (unsigned)combo::table_entry_bytes(rmax);
+    const unsigned dslot = dense ? round_up((unsigned)((p.N + dense_br - 1) / dense_br * (p.N + 2) * dense_br * 4), 128) : 0;
+    const unsigned entry = (unsigned)(plan.unw ? combo::entry_unw_bytes(rmax) : combo::table_entry_bytes(rmax));
     const unsigned long long slot_bytes = (unsigned long long)p.N * entry + dslot;
     int tab_slots = ((unsigned long long)p.S * slot_bytes <= 24u * 1024u && p.S >= 2) ? p.S : 2;
     unsigned table = round_up((unsigned)tab_slots * p.N * entry, 128) + (unsigned)tab_slots * dslot;
@@ -293,10 +295,10 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     return plan;
 }
 
-template <int EB, int GB, bool SGD, int RT>
+template <int EB, int GB, bool SGD, int RT, bool UNW = false>
 cudaError_t launch_staged_inst(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan,
                                cudaStream_t st) {
-    auto kern = combo::k_staged<EB, GB, SGD, RT>;
+    auto kern = combo::k_staged<EB, GB, SGD, RT, UNW>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem);
     if (e != cudaSuccess) return e;
     // Programmatic stream serialization: the kernel may be scheduled while the preceding
@@ -338,6 +340,21 @@ cudaError_t launch_staged_generic(const AggParams& p, const combo::TileMaps& map
     return launch_staged_inst<EB, GB, SGD, -1>(p, maps, plan, st);
 }
 
+// bfloat16 rows with unit weights
+template <int GB>
+cudaError_t launch_staged_unw(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan,
+                              cudaStream_t st) {
+    switch (plan.rt) {
+        case 1: return launch_staged_inst<2, GB, false, 1, true>(p, maps, plan, st);
+        case 2: return launch_staged_inst<2, GB, false, 2, true>(p, maps, plan, st);
+        case 3: return launch_staged_inst<2, GB, false, 3, true>(p, maps, plan, st);
+        case 4: return launch_staged_inst<2, GB, false, 4, true>(p, maps, plan, st);
+        case 8: return launch_staged_inst<2, GB, false, 8, true>(p, maps, plan, st);
+        case -2: return launch_staged_inst<2, GB, false, -2, true>(p, maps, plan, st);
+        default: return launch_staged_inst<2, GB, false, -1, true>(p, maps, plan, st);
+    }
+}
+
 cudaError_t launch_staged(const AggParams& p, const combo::TileMaps& maps, const StagedPlan& plan, int EB, bool sgd,
                           cudaStream_t st) {
     if (EB == 4) {
@@ -346,6 +363,7 @@ cudaError_t launch_staged(const AggParams& p, const combo::TileMaps& maps, const
         return sgd ? launch_staged_generic<4, 4, true>(p, maps, plan, st)
                    : launch_staged_generic<4, 4, false>(p, maps, plan, st);
     }
+    if (plan.unw) return plan.gb == 16 ? launch_staged_unw<16>(p, maps, plan, st) : launch_staged_unw<4>(p, maps, plan, st);
     if (plan.gb == 16) return launch_staged_r<2, 16, false>(p, maps, plan, st);
     if (plan.gb == 4) return launch_staged_r<2, 4, false>(p, maps, plan, st);
     return launch_staged_generic<2, 2, false>(p, maps, plan, st);
@@ -356,7 +374,7 @@ cudaError_t launch_staged(const AggParams& p, const combo::TileMaps& maps, const
 // take it (few rows: small tiles, many CTAs per SM).
 StagedPlan plan_tile(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, const DeviceInfo& dev,
                      bool* short_enough) {
-    StagedPlan plan = {false, 16, -1, 0, 0};
+    StagedPlan plan = {false, 16, -1, 0, 0, false};
     *short_enough = false;
     const int V = 16 / EB;
     const int narr = sgd ? 2 : 1;

@@ -55,21 +55,29 @@ __global__ void __launch_bounds__(256) k_pull_aggregate(const PullParams p) {
             // providers: the worker itself, then its peers ascending; a negative entry is a pull
             // that found no online peer (Section 4.2) and is skipped
             const int32_t* peers = my_idx + (size_t)l_lo * R;
+            // Eq. 3 as written: numerator in the fixed order, times the reciprocal of the
+            // denominator; a single provider is taken as it is
             float den = p.weights ? p.weights[w] : 1.0f;
+            int np = 1;
             for (int r = 0; r < R; ++r)
-                if (peers[r] >= 0) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
+                if (peers[r] >= 0) { den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f); ++np; }
             float acc[V], x[V];
             GroupLoad<EB, 16>::run(rows[w] + (size_t)c0 * EB, x);
-            float c = __fdiv_rn(p.weights ? p.weights[w] : 1.0f, den);
+            float c = (np == 1 || !p.weights) ? 1.0f : p.weights[w];
 #pragma unroll
             for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(c, x[i]);
             for (int r = 0; r < R; ++r) {
                 const int k = peers[r];
                 if (k < 0) continue;
                 GroupLoad<EB, 16>::run(rows[k] + (size_t)c0 * EB, x);
-                c = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                c = p.weights ? p.weights[k] : 1.0f;
 #pragma unroll
                 for (int i = 0; i < V; ++i) acc[i] = fmaf(c, x[i], acc[i]);
+            }
+            if (np > 1) {
+                const float scale = __fdiv_rn(1.0f, den);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(scale, acc[i]);
             }
             ElemOps<EB>::store_vec(orow + (size_t)c0 * EB, acc);
         } else {
@@ -77,16 +85,17 @@ __global__ void __launch_bounds__(256) k_pull_aggregate(const PullParams p) {
             for (long long col = c0; col < hi; ++col) {
                 const int32_t* peers = my_idx + (size_t)(col / p.L) * R;
                 float den = p.weights ? p.weights[w] : 1.0f;
+                int np = 1;
                 for (int r = 0; r < R; ++r)
-                    if (peers[r] >= 0) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
-                float acc = __fmul_rn(__fdiv_rn(p.weights ? p.weights[w] : 1.0f, den),
+                    if (peers[r] >= 0) { den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f); ++np; }
+                float acc = __fmul_rn((np == 1 || !p.weights) ? 1.0f : p.weights[w],
                                       ElemOps<EB>::load(rows[w] + (size_t)col * EB));
                 for (int r = 0; r < R; ++r) {
                     const int k = peers[r];
                     if (k < 0) continue;
-                    acc = fmaf(__fdiv_rn(p.weights ? p.weights[k] : 1.0f, den),
-                               ElemOps<EB>::load(rows[k] + (size_t)col * EB), acc);
+                    acc = fmaf(p.weights ? p.weights[k] : 1.0f, ElemOps<EB>::load(rows[k] + (size_t)col * EB), acc);
                 }
+                if (np > 1) acc = __fmul_rn(__fdiv_rn(1.0f, den), acc);
                 ElemOps<EB>::store(orow + (size_t)col * EB, acc);
             }
         }
@@ -260,8 +269,9 @@ __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStage
             }
             float den = p.weights ? p.weights[prov[0]] : 1.0f;
             for (int t = 1; t < np; ++t) den = __fadd_rn(den, p.weights ? p.weights[prov[t]] : 1.0f);
+            cf[entry_scale_word(RMAX)] = np == 1 ? 1.0f : __fdiv_rn(1.0f, den);
             for (int r = 0; r < np; ++r) {
-                cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[prov[r]] : 1.0f, den);
+                cf[2 * r] = cf[2 * r + 1] = (np == 1 || !p.weights) ? 1.0f : p.weights[prov[r]];
                 po[r] = (int)slot_of[prov[r]] * p.row_bytes;
             }
             for (int r = np; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }

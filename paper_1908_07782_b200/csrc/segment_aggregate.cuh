@@ -254,8 +254,7 @@ template <> struct PairStore<2, 16> {
 };
 // 32-bit streaming store executed only where `on` is non-zero (predicated, no branch)
 __device__ __forceinline__ void stcs_b32_if(unsigned char* p, uint32_t v, unsigned on) {
-    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; @q st.global.cs.b32 [%0], %1; }" ::"l"(p), "r"(v), "r"(on)
-                 : "memory");
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; @q st.global.cs.b32 [%0], %1; }" ::"l"(p), "r"(v), "r"(on));
 }
 template <> struct PairStore<4, 4> {
     __device__ static __forceinline__ void run(unsigned char* p, const f32x2 (&a)[2], unsigned mask) {
@@ -376,14 +375,18 @@ __device__ __noinline__ void direct_element(const AggParams& p, int w, long long
         first = false;
     }
     pi.rewind();
+    int np = 0;
+    for (int k = pi.next(); k >= 0; k = pi.next()) ++np;
+    pi.rewind();
     float acc = 0.0f;
     first = true;
     for (int k = pi.next(); k >= 0; k = pi.next()) {
-        const float cf = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+        const float cf = (np == 1 || !p.weights) ? 1.0f : p.weights[k];      // a single provider is taken as it is
         const float x = direct_x<EB, SGD>(p, k, c);
         acc = first ? __fmul_rn(cf, x) : fmaf(cf, x, acc);
         first = false;
     }
+    if (np > 1) acc = __fmul_rn(acc, __fdiv_rn(1.0f, den));
     ElemOps<EB>::store(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c) * EB, acc);
 }
 
@@ -396,9 +399,11 @@ __device__ __noinline__ void direct_element(const AggParams& p, int w, long long
 // naive order, in which the re-reads of a row are spread over the whole run and mostly come
 // from DRAM; kept as the contrast case for profiling.)
 //
-// Per block the providers and coefficients of the (at most two) segments it touches are
-// worked out once, into shared memory: slot s of [2][R+1] holds the provider list and the
-// coefficients of segment la + s, la = the segment of the block's first column.
+// Per block the providers and weights of the (at most two) segments it touches are worked
+// out once, into shared memory: slot s of [2][R+1] holds the provider list and the weights
+// |D_j| of segment la + s, la = the segment of the block's first column, and s_den[s] the
+// scale 1 / sum |D_j| (Eq. 3 as written: numerator in the fixed order, times the reciprocal
+// of the denominator; a single provider is taken as it is).
 template <int EB, bool SGD>
 __global__ void __launch_bounds__(256) k_direct(const AggParams p, long long blocks_per_row, int worker_major) {
     constexpr int V = ElemOps<EB>::V;
@@ -435,12 +440,12 @@ __global__ void __launch_bounds__(256) k_direct(const AggParams p, long long blo
                 }
             }
             s_np[sl] = np;
-            s_den[sl] = den;
+            s_den[sl] = np > 1 ? __fdiv_rn(1.0f, den) : 1.0f;
         }
         __syncthreads();
         for (int t = threadIdx.x; t < 2 * cap; t += 256) {
             const int sl = t / cap, r = t - sl * cap;
-            if (r < s_np[sl]) s_coef[t] = __fdiv_rn(p.weights ? p.weights[s_prov[t]] : 1.0f, s_den[sl]);
+            if (r < s_np[sl]) s_coef[t] = (s_np[sl] == 1 || !p.weights) ? 1.0f : p.weights[s_prov[t]];
         }
         __syncthreads();
         const long long g = blk * 256LL + threadIdx.x;
@@ -474,6 +479,9 @@ __global__ void __launch_bounds__(256) k_direct(const AggParams p, long long blo
                     for (int i = 0; i < V; ++i) acc[i] = fmaf(c, x[i], acc[i]);
                 }
             }
+            const float scale = s_den[sl];
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc[i] = __fmul_rn(scale, acc[i]);
             ElemOps<EB>::store_vec(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c0) * EB, acc);
         } else {
             for (long long c = lo; c < hi; ++c) {
@@ -488,6 +496,7 @@ __global__ void __launch_bounds__(256) k_direct(const AggParams p, long long blo
                     const float x = direct_x<EB, SGD>(p, prov[r], c);
                     acc = r == 0 ? __fmul_rn(coef[r], x) : fmaf(coef[r], x, acc);
                 }
+                acc = __fmul_rn(s_den[sl], acc);
                 ElemOps<EB>::store(p.out + ((size_t)w * (size_t)p.pitch + (size_t)c) * EB, acc);
             }
         }
@@ -636,24 +645,34 @@ __device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t& phase, in
     return ok;
 }
 
-// Coefficient table entry of one (slot, row): c2[RMAX+1] coefficients, each already
-// duplicated into a binary32 pair, then poff[RMAX+1] ints (shared-memory byte offset
-// of each provider's staged row inside a box block, its phase included); padded to 16.
-__host__ __device__ constexpr int table_entry_bytes(int rmax) { return ((rmax + 1) * 12 + 15) / 16 * 16; }
+// Eq. 3 is evaluated as it is written: the numerator sum |D_j| x_j is accumulated over the
+// providers in the fixed order (the first term a product, the others fused multiply-adds),
+// and the result is the numerator times the binary32 reciprocal of the denominator, which
+// is summed in the same order.  A single provider is taken as it is (weight and scale 1).
+//
+// Coefficient table entry of one (slot, row): c2[RMAX+1] weights |D_j| of the providers,
+// each already duplicated into a binary32 pair, then poff[RMAX+1] ints (shared-memory byte
+// offset of each provider's staged row inside a box block, its phase included), then the
+// scale 1 / sum |D_j| as one float; padded to 16.
+__host__ __device__ constexpr int table_entry_bytes(int rmax) { return ((rmax + 1) * 12 + 4 + 15) / 16 * 16; }
+__host__ __device__ constexpr int entry_scale_word(int rmax) { return 3 * (rmax + 1); }
 
 template <int RMAX>
 struct RowCtx {
-    f32x2 c2[RMAX + 1];    // coefficient of each provider, duplicated into a pair
+    f32x2 c2[RMAX + 1];    // weight of each provider, duplicated into a pair
     int poff[RMAX + 1];
+    f32x2 s2;              // the scale, duplicated
 };
 
+// `entry` is the entry's shared-window address; it is read as whole 128-bit vectors exactly
+// once (through the generic pointer the compiler fetched some coefficient pairs a second time).
 template <int RMAX>
-__device__ __forceinline__ void load_entry(const unsigned char* entry, RowCtx<RMAX>& c) {
+__device__ __forceinline__ void load_entry(uint32_t entry, RowCtx<RMAX>& c) {
     constexpr int ENT = table_entry_bytes(RMAX);
     uint32_t raw[ENT / 4];
 #pragma unroll
     for (int i = 0; i < ENT / 16; ++i) {
-        const uint4 v = reinterpret_cast<const uint4*>(entry)[i];
+        const uint4 v = lds128(entry + 16 * i);
         raw[4 * i] = v.x; raw[4 * i + 1] = v.y; raw[4 * i + 2] = v.z; raw[4 * i + 3] = v.w;
     }
 #pragma unroll
@@ -661,6 +680,7 @@ __device__ __forceinline__ void load_entry(const unsigned char* entry, RowCtx<RM
         c.c2[r] = pair_bits(raw[2 * r], raw[2 * r + 1]);
         c.poff[r] = (int)raw[2 * (RMAX + 1) + r];
     }
+    c.s2 = pair_bits(raw[entry_scale_word(RMAX)], raw[entry_scale_word(RMAX)]);
 }
 
 // One lane's share of an item (512 bytes of an output row): self first, then the
@@ -683,6 +703,8 @@ __device__ __forceinline__ void item_fast(uint32_t base, const RowCtx<RMAX>& c, 
             for (int i = 0; i < NP; ++i) acc[i] = fma2(c.c2[r], x[i], acc[i]);
         }
     }
+#pragma unroll
+    for (int i = 0; i < NP; ++i) acc[i] = mul2(c.s2, acc[i]);
     PairStore<EB, GB>::run(outp, acc, mask);
 }
 
@@ -703,6 +725,127 @@ __device__ __forceinline__ void item_box(uint32_t base, const RowCtx<RMAX>& c, i
             for (int i = 0; i < NP; ++i) acc[i] = fma2(c.c2[r], x[i], acc[i]);
         }
     }
+#pragma unroll
+    for (int i = 0; i < NP; ++i) acc[i] = mul2(c.s2, acc[i]);
+    PairStoreBox<EB, GB>::template run<LAST>(outp, acc, last_on);
+}
+
+// ---- bfloat16 rows with unit weights (weights == NULL) --------------------------------
+// The numerator of Eq. 3 is then the plain sum of the providers' values in the fixed order,
+// and sm_100 adds a bfloat16 operand to a binary32 one in a single instruction
+// (add.rn.f32.bf16: the bfloat16 value is widened exactly, one rounding, either half of a
+// 32-bit register) -- the same result as widening first and adding, without the two integer
+// instructions per packed word that the widening costs.  Entries need no weights:
+// poff[RMAX+1], the scale 1 / np as one float, np = number of providers; padded to 16.
+// Providers are packed into the first np slots; the others are never read.
+__host__ __device__ constexpr int entry_unw_bytes(int rmax) { return ((rmax + 1) * 4 + 8 + 15) / 16 * 16; }
+
+template <int RMAX>
+struct RowCtxU {
+    int poff[RMAX + 1];
+    f32x2 s2;
+    int np;
+};
+template <int RMAX, bool UNW> struct CtxSel { typedef RowCtx<RMAX> type; };
+template <int RMAX> struct CtxSel<RMAX, true> { typedef RowCtxU<RMAX> type; };
+template <int RMAX, bool UNW> __host__ __device__ constexpr int entry_bytes_of() {
+    return UNW ? entry_unw_bytes(RMAX) : table_entry_bytes(RMAX);
+}
+
+template <int RMAX>
+__device__ __forceinline__ void load_entry(uint32_t entry, RowCtxU<RMAX>& c) {
+    constexpr int ENT = entry_unw_bytes(RMAX);
+    uint32_t raw[ENT / 4];
+#pragma unroll
+    for (int i = 0; i < ENT / 16; ++i) {
+        const uint4 v = lds128(entry + 16 * i);
+        raw[4 * i] = v.x; raw[4 * i + 1] = v.y; raw[4 * i + 2] = v.z; raw[4 * i + 3] = v.w;
+    }
+#pragma unroll
+    for (int r = 0; r <= RMAX; ++r) c.poff[r] = (int)raw[r];
+    c.s2 = pair_bits(raw[RMAX + 1], raw[RMAX + 1]);
+    c.np = (int)raw[RMAX + 2];
+}
+
+// binary32 + bfloat16 from the low / the high half of a packed word
+__device__ __forceinline__ float add_bf16_lo(uint32_t w, float c) {
+    const unsigned short h = (unsigned short)(w & 0xffffu);
+    asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(c) : "h"(h));
+    return c;
+}
+__device__ __forceinline__ float add_bf16_hi(uint32_t w, float c) {
+    const unsigned short h = (unsigned short)(w >> 16);
+    asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(c) : "h"(h));
+    return c;
+}
+
+// the four packed words of a lane's share of an item
+template <int GB> struct WordLoad;
+template <> struct WordLoad<16> {
+    __device__ static __forceinline__ void run(uint32_t a, uint32_t (&w)[4]) {
+        const uint4 v = lds128(a);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    }
+};
+template <> struct WordLoad<4> {
+    __device__ static __forceinline__ void run(uint32_t a, uint32_t (&w)[4]) {
+        w[0] = lds32<0>(a); w[1] = lds32<128>(a); w[2] = lds32<256>(a); w[3] = lds32<384>(a);
+    }
+};
+
+// Sum of the providers' values in the fixed order, times the scale: a lane's share of an item.
+template <int GB, int RMAX, bool FIXED_R>
+__device__ __forceinline__ void sum_unw(uint32_t base, const RowCtxU<RMAX>& c, f32x2 (&acc)[4]) {
+    uint32_t w[4];
+    float a[8];
+    WordLoad<GB>::run(base + c.poff[0], w);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        a[2 * i] = __uint_as_float(w[i] << 16);
+        a[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+    if (FIXED_R && c.np == RMAX + 1) {
+        // all replicas present (the usual case): straight-line code
+#pragma unroll
+        for (int r = 1; r <= RMAX; ++r) {
+            WordLoad<GB>::run(base + c.poff[r], w);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                a[2 * i] = add_bf16_lo(w[i], a[2 * i]);
+                a[2 * i + 1] = add_bf16_hi(w[i], a[2 * i + 1]);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int r = 1; r <= RMAX; ++r) {
+            if (r < c.np) {
+                WordLoad<GB>::run(base + c.poff[r], w);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    a[2 * i] = add_bf16_lo(w[i], a[2 * i]);
+                    a[2 * i + 1] = add_bf16_hi(w[i], a[2 * i + 1]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        acc[i] = mul2(c.s2, pair_bits(__float_as_uint(a[2 * i]), __float_as_uint(a[2 * i + 1])));
+}
+template <int EB, int GB, int RMAX, bool FIXED_R>
+__device__ __forceinline__ void item_fast(uint32_t base, const RowCtxU<RMAX>& c, int, unsigned char* outp,
+                                          unsigned mask) {
+    static_assert(EB == 2 && (GB == 16 || GB == 4), "bfloat16 only");
+    f32x2 acc[4];
+    sum_unw<GB, RMAX, FIXED_R>(base, c, acc);
+    PairStore<EB, GB>::run(outp, acc, mask);
+}
+template <int EB, int GB, int RMAX, bool FIXED_R, bool LAST>
+__device__ __forceinline__ void item_box(uint32_t base, const RowCtxU<RMAX>& c, int, unsigned char* outp,
+                                         bool last_on) {
+    static_assert(EB == 2 && GB == 4, "bfloat16 word mode only");
+    f32x2 acc[4];
+    sum_unw<GB, RMAX, FIXED_R>(base, c, acc);
     PairStoreBox<EB, GB>::template run<LAST>(outp, acc, last_on);
 }
 
@@ -724,10 +867,10 @@ __device__ __forceinline__ void sgd_step_in_place(unsigned char* stage, int byte
 
 // Coefficient / offset table of `nslots` consecutive segments starting at l0_build, built by
 // `nthreads` threads of which the caller is number t: entry [slot][w] of ENT bytes.
-template <int EB, int RMAX>
+template <int EB, int RMAX, bool UNW = false>
 __device__ __forceinline__ void build_coef_table(const AggParams& p, unsigned char* tab, int R, int l0_build,
                                                  int nslots, int t, int nthreads) {
-    constexpr int ENT = table_entry_bytes(RMAX);
+    constexpr int ENT = entry_bytes_of<RMAX, UNW>();
     const int N = p.N;
     for (int q = t; q < nslots * N; q += nthreads) {
         const int slot = q / N, w = q - slot * N;
@@ -735,7 +878,7 @@ __device__ __forceinline__ void build_coef_table(const AggParams& p, unsigned ch
         if (l < p.S) {
             const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
             float* cf = reinterpret_cast<float*>(tab + ((size_t)slot * N + w) * ENT);   // pairs
-            int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
+            int* po = UNW ? reinterpret_cast<int*>(cf) : reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
             // providers in the fixed order: the worker itself (unless it is a newcomer), then
             // the peers ascending; a negative entry is a pull that found no online peer
             int prov[RMAX + 1];
@@ -748,9 +891,17 @@ __device__ __forceinline__ void build_coef_table(const AggParams& p, unsigned ch
             if (np == 0) prov[np++] = w;                 // nothing to aggregate: keep the own values
             float den = p.weights ? p.weights[prov[0]] : 1.0f;
             for (int i = 1; i < np; ++i) den = __fadd_rn(den, p.weights ? p.weights[prov[i]] : 1.0f);
+            // a single provider is taken as it is
+            const float scale = np == 1 ? 1.0f : __fdiv_rn(1.0f, den);
+            if (UNW) {
+                cf[RMAX + 1] = scale;
+                po[RMAX + 2] = np;
+            } else {
+                cf[entry_scale_word(RMAX)] = scale;
+            }
             for (int r = 0; r < np; ++r) {
                 const int k = prov[r];
-                cf[2 * r] = cf[2 * r + 1] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+                if (!UNW) cf[2 * r] = cf[2 * r + 1] = (np == 1 || !p.weights) ? 1.0f : p.weights[k];
                 // staged row of worker k: classes are stored one after another
                 const int jk = k % p.m;
                 int base = 0;
@@ -758,8 +909,11 @@ __device__ __forceinline__ void build_coef_table(const AggParams& p, unsigned ch
                 const int phase = (int)(((long long)k * p.pitch * EB) & 15);
                 po[r] = (base + k / p.m) * p.row_bytes + phase;
             }
-            // unused slots: coefficient zero on a row that is known to hold finite values
-            for (int r = np; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
+            // unused slots: weight zero on a row that is known to hold finite values
+            for (int r = np; r <= RMAX; ++r) {
+                if (!UNW) cf[2 * r] = cf[2 * r + 1] = 0.0f;
+                po[r] = po[0];
+            }
         }
     }
 }
@@ -816,9 +970,9 @@ template <int EB> struct DenseRows {
     static constexpr int CH = 1;                     // 512-byte chunks a unit spans
 };
 
-// Dense coefficient blocks of `nslots` segments: [slot][block][k = 0..N][BR] floats; k < N:
-// coefficient of staged row k for output row BR*block + b, zero if it is not a provider or is
-// the output row itself; k = N: the output row's own coefficient.
+// Dense coefficient blocks of `nslots` segments: [slot][block][k = 0..N+1][BR] floats; k < N:
+// weight |D_k| of staged row k for output row BR*block + b, zero if it is not a provider or is
+// the output row itself; k = N: the output row's own weight; k = N + 1: its scale 1 / sum.
 template <int EB>
 __device__ __forceinline__ void build_dense_table(const AggParams& p, unsigned char* dtab, int R, int l0_build,
                                                   int nslots, int t, int nthreads) {
@@ -830,17 +984,20 @@ __device__ __forceinline__ void build_dense_table(const AggParams& p, unsigned c
         const int l = l0_build + slot;
         if (l >= p.S) continue;
         float* col = reinterpret_cast<float*>(dtab + (size_t)slot * p.dslot_bytes) +
-                     (size_t)(w / BR) * (N + 1) * BR + (w % BR);
-        for (int k = 0; k <= N; ++k) col[(size_t)k * BR] = 0.0f;
+                     (size_t)(w / BR) * (N + 2) * BR + (w % BR);
+        for (int k = 0; k <= N + 1; ++k) col[(size_t)k * BR] = 0.0f;
         if (w >= N) continue;
         const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)l) * (size_t)R;
         float den = p.weights ? p.weights[w] : 1.0f;
+        int np = 1;
         for (int r = 0; r < R; ++r)
-            if (peers[r] >= 0) den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f);
-        col[(size_t)N * BR] = __fdiv_rn(p.weights ? p.weights[w] : 1.0f, den);
+            if (peers[r] >= 0) { den = __fadd_rn(den, p.weights ? p.weights[peers[r]] : 1.0f); ++np; }
+        // a single provider is taken as it is
+        col[(size_t)N * BR] = (np == 1 || !p.weights) ? 1.0f : p.weights[w];
+        col[(size_t)(N + 1) * BR] = np == 1 ? 1.0f : __fdiv_rn(1.0f, den);
         for (int r = 0; r < R; ++r) {
             const int k = peers[r];
-            if (k >= 0) col[(size_t)k * BR] = __fdiv_rn(p.weights ? p.weights[k] : 1.0f, den);
+            if (k >= 0) col[(size_t)k * BR] = p.weights ? p.weights[k] : 1.0f;
         }
     }
 }
@@ -878,7 +1035,7 @@ __device__ __forceinline__ void aggregate_dense(const AggParams& p, uint32_t sta
         const int w0 = blk * BR;
         const int col_off = gi * CH * 512 + lane * 16;                 // byte offset inside the box payload
         const uint32_t base = stage_s + xb * block_bytes + col_off;
-        uint32_t ct = dt_s + (uint32_t)(blk * (N + 1) * BR * 4);
+        uint32_t ct = dt_s + (uint32_t)(blk * (N + 2) * BR * 4);
         f32x2 acc[BR][CH * NP], x[CH * NP], c[BR];
         // own terms first
         dense_coefs<BR>(ct + (uint32_t)(N * BR * 4), c);
@@ -912,9 +1069,13 @@ __device__ __forceinline__ void aggregate_dense(const AggParams& p, uint32_t sta
             xa += p.row_bytes;
             ct += BR * 4;
         }
+        // ct now points at row N (the own weights); the scales follow
+        dense_coefs<BR>(ct + (uint32_t)(BR * 4), c);
         unsigned char* o = p.out + (size_t)w0 * pitch_bytes + (size_t)t0 * EB + (size_t)xb * box_payload + col_off;
 #pragma unroll
         for (int b = 0; b < BR; ++b) {
+#pragma unroll
+            for (int i = 0; i < CH * NP; ++i) acc[b][i] = mul2(c[b], acc[b][i]);
             if (w0 + b < N) {
 #pragma unroll
                 for (int h = 0; h < CH; ++h) {
@@ -932,14 +1093,15 @@ __device__ __forceinline__ void aggregate_dense(const AggParams& p, uint32_t sta
 // stored to the output rows.  `stage` holds the tile (its shared-window address is stage_s),
 // tab0 the table entries of segment l0 (those of l0 + 1 follow them), m_bnd is the local
 // column where segment l0 + 1 starts.
-template <int EB, int GB, int RT>
+template <int EB, int GB, int RT, bool UNW = false>
 __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpShare<EB, GB>& ws,
                                                const unsigned char* stage, uint32_t stage_s,
                                                const unsigned char* tab0, long long tile, long long m_bnd,
                                                int lane, const unsigned char* dtab0 = nullptr) {
     constexpr int V = ElemOps<EB>::V;
     constexpr int RMAX = rmax_of(RT);
-    constexpr int ENT = table_entry_bytes(RMAX);
+    constexpr int ENT = entry_bytes_of<RMAX, UNW>();
+    typedef typename CtxSel<RMAX, UNW>::type Ctx;
     constexpr int CPB = WarpShare<EB, GB>::CPB;
     constexpr int PIECES = WarpShare<EB, GB>::PIECES;
     constexpr int PSTRIDE = WarpShare<EB, GB>::PSTRIDE;
@@ -952,6 +1114,7 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
     const long long t0 = tile * (long long)p.T;
     const long long t1 = (t0 + p.T < p.width) ? t0 + p.T : p.width;
     const bool interior = (m_bnd >= t1) && (t0 + p.T <= p.width);   // one segment, whole tile
+    const uint32_t tab_s = smem_u32(tab0);
     if constexpr (RT == -3 && GB == 16) {
         if (interior) {
             aggregate_dense<EB>(p, stage_s, dtab0, t0, ws.cw, ws.nwarps, lane);
@@ -964,16 +1127,28 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
         // word mode: a unit is a whole row of a box, and only the last piece of it can lie
         // outside the box's payload (a loop-invariant lane predicate)
         if constexpr (GB < 16) {
-            RowCtx<RMAX> c;
+            Ctx c;
             const uint32_t lane_base = stage_s + lane * GB;
             const bool last_on = (CPB - 1) * 512 + lane * GB + (PIECES - 1) * PSTRIDE < box_payload;
             if (p.nbx == 1) {
                 // the tile is one box (many rows): a unit is a row
-                const unsigned char* ent = tab0 + (size_t)u_begin * ENT;
+                uint32_t ent = tab_s + (uint32_t)(u_begin * ENT);
                 unsigned char* orow = p.out + (size_t)u_begin * pitch_bytes + (size_t)t0 * EB + lane * GB;
+                // The entry of the next row is fetched while this row is worked on (the last
+                // fetch reads the entry behind the warp's rows: inside the table or the stage
+                // ring, never used).
+                // (Not with the wide entries of the many-replica kernels: they would spill.)
+                constexpr bool AHEAD = RMAX <= 8;
+                typename CtxSel<AHEAD ? RMAX : 0, UNW>::type c_next;
+                if constexpr (AHEAD) load_entry<RMAX>(ent, c_next);
 #pragma unroll 4   // measured: 2 -> 4 gains 1.7 % with 128 bf16 rows, 8 gains nothing
                 for (int u = u_begin; u < u_end; ++u) {
-                    load_entry<RMAX>(ent, c);
+                    if constexpr (AHEAD) {
+                        c = c_next;
+                        load_entry<RMAX>(ent + ENT, c_next);
+                    } else {
+                        load_entry<RMAX>(ent, c);
+                    }
 #pragma unroll
                     for (int ch = 0; ch < CPB - 1; ++ch)
                         item_box<EB, GB, RMAX, (RT >= 0), false>(lane_base + ch * 512, c, R, orow + ch * 512, true);
@@ -985,7 +1160,7 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
             } else {
                 // several boxes per tile (few rows): rows outside, boxes inside
                 const int nbx = p.nbx;
-                const unsigned char* ent = tab0 + (size_t)row * ENT;
+                uint32_t ent = tab_s + (uint32_t)(row * ENT);
                 unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
                 int u = u_begin;
                 while (u < u_end) {
@@ -1009,21 +1184,21 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
         // quarter-kilobyte row pieces (so many rows that wider ones do not fit): a warp takes
         // two rows at a time, one per half-warp, each lane its 16 bytes
         const int half = lane >> 4, hl = lane & 15;
-        RowCtx<RMAX> c;
+        Ctx c;
         const uint32_t lane_base = stage_s + hl * 16;
         unsigned char* ocol = p.out + (size_t)t0 * EB + hl * 16;
         for (int u = u_begin; u < u_end; u += 2) {
             const int myrow = u + half;
             if (myrow < u_end && hl * 16 < box_payload) {
-                load_entry<RMAX>(tab0 + (size_t)myrow * ENT, c);
+                load_entry<RMAX>(tab_s + (uint32_t)(myrow * ENT), c);
                 item_fast<EB, GB, RMAX, (RT >= 0)>(lane_base, c, R, ocol + (size_t)myrow * pitch_bytes, 0xffu);
             }
         }
     } else if (interior) {
         // every unit is whole and lies in segment l0: the lean loop, rows outside, boxes inside
-        RowCtx<RMAX> c;
+        Ctx c;
         const int nbx = p.nbx;
-        const unsigned char* ent = tab0 + (size_t)row * ENT;
+        uint32_t ent = tab_s + (uint32_t)(row * ENT);
         unsigned char* orow = p.out + (size_t)row * pitch_bytes + (size_t)t0 * EB + lane * GB;
         const uint32_t lane_base = stage_s + lane * GB;
         int u = u_begin;
@@ -1056,8 +1231,8 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
                     const bool whole = c0 + V <= p.width;
                     const bool one_seg = (c0 + V <= m_bnd) || (c0 >= m_bnd);
                     if (whole && one_seg) {
-                        RowCtx<RMAX> cc;
-                        load_entry<RMAX>(tab0 + ((size_t)(c0 >= m_bnd ? 1 : 0) * N + row) * ENT, cc);
+                        Ctx cc;
+                        load_entry<RMAX>(tab_s + (uint32_t)(((c0 >= m_bnd ? 1 : 0) * N + row) * ENT), cc);
                         item_fast<EB, GB, RMAX, (RT >= 0)>(
                             ubase, cc, R, p.out + (size_t)row * pitch_bytes + (size_t)c0 * EB, 0xffu);
                         done = true;
@@ -1074,11 +1249,21 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
                             if (col >= p.width) continue;
                             const unsigned char* ent = tab0 + ((size_t)(col >= m_bnd ? 1 : 0) * N + row) * ENT;
                             const float* cf = reinterpret_cast<const float*>(ent);       // pairs
-                            const int* po = reinterpret_cast<const int*>(cf + 2 * (RMAX + 1));
                             const unsigned char* eb = stage + xb * block_bytes + pin + e * EB;
-                            float acc = __fmul_rn(cf[0], ElemOps<EB>::load(eb + po[0]));
-                            for (int r = 1; r <= R; ++r)
-                                acc = fmaf(cf[2 * r], ElemOps<EB>::load(eb + po[r]), acc);
+                            float acc;
+                            if constexpr (UNW) {
+                                const int* po = reinterpret_cast<const int*>(ent);
+                                const int np = po[RMAX + 2];
+                                acc = ElemOps<EB>::load(eb + po[0]);
+                                for (int r = 1; r < np; ++r) acc = __fadd_rn(ElemOps<EB>::load(eb + po[r]), acc);
+                                acc = __fmul_rn(cf[RMAX + 1], acc);
+                            } else {
+                                const int* po = reinterpret_cast<const int*>(cf + 2 * (RMAX + 1));
+                                acc = __fmul_rn(cf[0], ElemOps<EB>::load(eb + po[0]));
+                                for (int r = 1; r <= R; ++r)
+                                    acc = fmaf(cf[2 * r], ElemOps<EB>::load(eb + po[r]), acc);
+                                acc = __fmul_rn(cf[entry_scale_word(RMAX)], acc);
+                            }
                             ElemOps<EB>::store(p.out + (size_t)row * pitch_bytes + (size_t)col * EB, acc);
                         }
                     }
@@ -1089,13 +1274,13 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
     }
 }
 
-template <int EB, int GB, bool SGD, int RT>
+template <int EB, int GB, bool SGD, int RT, bool UNW = false>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     // RT: the number of replicas the kernel is specialised on, -1 = any up to kGenericR,
-    // -2 = any up to kStagedMaxR
+    // -2 = any up to kStagedMaxR.  UNW: bfloat16 rows with unit weights (see RowCtxU).
     constexpr int RMAX = rmax_of(RT);
-    constexpr int ENT = table_entry_bytes(RMAX);
+    constexpr int ENT = entry_bytes_of<RMAX, UNW>();
     extern __shared__ __align__(128) unsigned char smem[];
     StagedHeader* hdr = reinterpret_cast<StagedHeader*>(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1255,11 +1440,11 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
     unsigned char* dtab = smem + p.dtab_off;               // dense coefficient blocks, one set per table slot
     if ((long long)blockIdx.x < p.n_tiles) {
         if (whole_table) {
-            build_coef_table<EB, RMAX>(p, tab, R, 0, p.S, ctid, kConsumerThreads);
+            build_coef_table<EB, RMAX, UNW>(p, tab, R, 0, p.S, ctid, kConsumerThreads);
             if (DENSE) build_dense_table<EB>(p, dtab, R, 0, p.S, ctid, kConsumerThreads);
         } else {
             cached_l0 = (int)((p.p_begin + (long long)blockIdx.x * p.T) / p.L);
-            build_coef_table<EB, RMAX>(p, tab, R, cached_l0, 2, ctid, kConsumerThreads);
+            build_coef_table<EB, RMAX, UNW>(p, tab, R, cached_l0, 2, ctid, kConsumerThreads);
             if (DENSE) build_dense_table<EB>(p, dtab, R, cached_l0, 2, ctid, kConsumerThreads);
         }
         if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(7); return; }
@@ -1282,7 +1467,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
         if (!whole_table && m_l0 != cached_l0) {
             // table for segments l0 and l0+1 (rebuilt at most S times per CTA)
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(4); return; }
-            build_coef_table<EB, RMAX>(p, tab, R, m_l0, 2, ctid, kConsumerThreads);
+            build_coef_table<EB, RMAX, UNW>(p, tab, R, m_l0, 2, ctid, kConsumerThreads);
             if (DENSE) build_dense_table<EB>(p, dtab, R, m_l0, 2, ctid, kConsumerThreads);
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(5); return; }
             cached_l0 = m_l0;
@@ -1294,7 +1479,7 @@ k_staged(const AggParams p, const __grid_constant__ TileMaps maps) {
             if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(6); return; }
         }
 
-        aggregate_tile<EB, GB, RT>(p, ws, stage, stage_s, tab0, tile, m_bnd, lane,
+        aggregate_tile<EB, GB, RT, UNW>(p, ws, stage, stage_s, tab0, tile, m_bnd, lane,
                                    DENSE ? dtab + (size_t)(whole_table ? m_l0 : 0) * p.dslot_bytes : nullptr);
 
         // The fused step rewrote the stage with ordinary stores; the copy that refills it goes

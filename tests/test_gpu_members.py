@@ -38,9 +38,16 @@ CASES = [(8, 40_000, 4, 2, torch.float32), (13, 50_001, 5, 4, torch.float32), (3
          (24, 40_000, 4, 10, torch.float32), (30, 24_000, 5, 12, torch.bfloat16)]    # many replicas
 
 
-@pytest.mark.parametrize("N,P,S,R,dtype", CASES)
+# unit weights (no weights array) take kernels of their own for bfloat16 rows: the sum of the
+# providers' values by mixed-precision adds, with the provider count in the table entry
+CASES_UNIT = [(128, 5_002, 16, 4, torch.bfloat16), (20, 30_000, 3, 6, torch.bfloat16),
+              (16, 40_008, 4, 4, torch.bfloat16), (30, 24_000, 5, 12, torch.bfloat16),
+              (13, 50_001, 5, 4, torch.float32)]
+
+
+@pytest.mark.parametrize("N,P,S,R,dtype,weighted", [c + (True,) for c in CASES] + [c + (False,) for c in CASES_UNIT])
 @pytest.mark.parametrize("path", [combo.PATH_DIRECT, combo.PATH_STAGED])
-def test_aggregate_members(N, P, S, R, dtype, path):
+def test_aggregate_members(N, P, S, R, dtype, weighted, path):
     rng = np.random.default_rng(N + P)
     g = torch.Generator().manual_seed(N)
     x = (torch.randn(N, P, generator=g) * 0.05 + 0.01).to(dtype)
@@ -57,8 +64,9 @@ def test_aggregate_members(N, P, S, R, dtype, path):
     veteran = [int(v) for v in online if not newcomer[v]]
     idx_np[veteran[-1], 0, :] = -1                             # a segment with no peer at all
     xb = to_bits(x)
-    exact = oracle.segment_aggregate_members(xb, idx_np, S, R, w.numpy(), newcomer)
-    ordered = oracle.segment_aggregate_members(xb, idx_np, S, R, w.numpy(), newcomer, ordered=True)
+    wn = w.numpy() if weighted else None
+    exact = oracle.segment_aggregate_members(xb, idx_np, S, R, wn, newcomer)
+    ordered = oracle.segment_aggregate_members(xb, idx_np, S, R, wn, newcomer, ordered=True)
     # on the device the newcomers' rows hold NaN: they must never be read
     xd = x.clone()
     xd[torch.from_numpy(newcomer.astype(bool))] = float("nan")
@@ -67,7 +75,8 @@ def test_aggregate_members(N, P, S, R, dtype, path):
     idx = torch.from_numpy(idx_np).to(DEV)
     combo.combo_set_kernel_path(path)
     try:
-        combo.combo_segment_aggregate_members(xd, out, w.to(DEV), idx, newcomer.tolist(), N, P, S, R)
+        combo.combo_segment_aggregate_members(xd, out, w.to(DEV) if weighted else None, idx, newcomer.tolist(),
+                                              N, P, S, R)
         torch.cuda.synchronize()
     finally:
         combo.combo_set_kernel_path(combo.PATH_AUTO)
