@@ -641,25 +641,49 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
         p.coef_off = header;
         p.rowoff_off = p.coef_off + round_up((unsigned)N * 4u, 128);
         p.part_off = p.rowoff_off + round_up((unsigned)N * 4u, 128);
-        p.mean_off = p.part_off + 2u * combo::kConsumerThreads * V * 4u;   // two copies of G * PSTR floats
-        p.stage_off = p.mean_off + 2u * combo::kDivTile * 4u;
         p.m = m;
-        const long long budget = (long long)dev->smem_optin - p.stage_off - 256;
+        // shared memory in front of the stages for a box of c columns.  Vector mode: two copies
+        // of G * PSTR floats of partial sums and two of the widest tile's means.  Word mode: two
+        // copies of [consumer warps][words per row rounded up to a power of two] sums and two
+        // of 256 means.
+        auto front = [&](int c) {
+            unsigned part, mean;
+            if (word) {
+                const int nu = (c - V) * EB / 4;
+                int nup = 16;
+                while (nup < nu) nup <<= 1;
+                part = 2u * combo::kConsumerWarps * (unsigned)(nup * (4 / EB)) * 4u;
+                mean = 2u * combo::kDivWordMeans * 4u;
+            } else {
+                part = 2u * combo::kConsumerThreads * V * 4u;
+                mean = 2u * combo::kDivTile * 4u;
+            }
+            p.mean_off = p.part_off + part;
+            p.stage_off = p.mean_off + mean;
+            return (long long)dev->smem_optin - p.stage_off - 256;
+        };
         // tile: the widest whose stage stays within 64 KB (at least 64 columns if two stages
         // fit at all); tiles beyond 256 columns are made of 256-column boxes.  With row phases
-        // one box of at most 256 columns.
+        // one box of at most 256 columns: the widest of which three stages fit (the consumers
+        // then hold two tiles at a time and need one barrier per tile), else the widest of
+        // which two fit.
         int TC = 0, box = 0;
+        bool pipe = !word;
         if (word) {
-            for (int c = combo::kDivBox; c >= 64; c >>= 1)
-                if (2LL * p.narr * N * c * EB <= budget) { TC = c - V; box = c; break; }
+            for (int need = 3; need >= 2 && TC == 0; --need)
+                for (int c = combo::kDivBox; c >= 64; c >>= 1) {
+                    if (t_tile > 0 && c != t_tile) continue;
+                    if ((long long)need * p.narr * N * c * EB <= front(c)) { TC = c - V; box = c; pipe = need == 3; break; }
+                }
         } else {
             for (int c = combo::kDivTile; c >= 64; c >>= 1) {
                 const long long stage = (long long)p.narr * N * c * EB;
-                if (2 * stage > budget || p.narr * (c > combo::kDivBox ? c / combo::kDivBox : 1) > 32) continue;
+                if (2 * stage > front(c) || p.narr * (c > combo::kDivBox ? c / combo::kDivBox : 1) > 32) continue;
                 if (stage <= 64 * 1024 || c == 64 || c <= combo::kDivBox) { TC = c; break; }
             }
             box = TC > combo::kDivBox ? combo::kDivBox : TC;
         }
+        const long long budget = TC > 0 ? front(box) : 0;
         combo::TileMaps maps;
         bool ok = TC > 0;
         for (int a = 0; ok && a < p.narr; ++a)
@@ -680,20 +704,24 @@ combo_status divergence_impl(const void* models, const void* mean_of, int EB, co
             nblocks = (int)(p.n_tiles < dev->sms ? p.n_tiles : dev->sms);
             const size_t smem = (size_t)p.stage_off + (size_t)stages * p.stage_bytes + 16;
             cudaError_t e = cudaErrorInvalidValue;
-#define COMBO_DIV_LAUNCH(EBV, TCV, WV)                                                                          \
-    if (EB == EBV && TC == TCV && word == WV) {                                                                 \
-        e = cudaFuncSetAttribute(combo::k_divergence_staged<EBV, TCV, WV>,                                      \
+#define COMBO_DIV_LAUNCH_P(EBV, TCV, WV, PV)                                                                    \
+    if (EB == EBV && TC == TCV && word == WV && pipe == PV) {                                                   \
+        e = cudaFuncSetAttribute(combo::k_divergence_staged<EBV, TCV, WV, PV>,                                  \
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);                       \
         if (e == cudaSuccess)                                                                                   \
-            combo::k_divergence_staged<EBV, TCV, WV><<<nblocks, combo::kStagedThreads, smem, st>>>(p, maps);    \
+            combo::k_divergence_staged<EBV, TCV, WV, PV><<<nblocks, combo::kStagedThreads, smem, st>>>(p, maps); \
     }
+#define COMBO_DIV_LAUNCH(EBV, TCV, WV) COMBO_DIV_LAUNCH_P(EBV, TCV, WV, true)
+#define COMBO_DIV_LAUNCH_W(EBV, TCV) COMBO_DIV_LAUNCH_P(EBV, TCV, true, true) COMBO_DIV_LAUNCH_P(EBV, TCV, true, false)
             COMBO_DIV_LAUNCH(4, 1024, false) COMBO_DIV_LAUNCH(4, 512, false)
             COMBO_DIV_LAUNCH(2, 1024, false) COMBO_DIV_LAUNCH(2, 512, false)
             COMBO_DIV_LAUNCH(4, 256, false) COMBO_DIV_LAUNCH(4, 128, false) COMBO_DIV_LAUNCH(4, 64, false)
             COMBO_DIV_LAUNCH(2, 256, false) COMBO_DIV_LAUNCH(2, 128, false) COMBO_DIV_LAUNCH(2, 64, false)
-            COMBO_DIV_LAUNCH(4, 252, true) COMBO_DIV_LAUNCH(4, 124, true) COMBO_DIV_LAUNCH(4, 60, true)
-            COMBO_DIV_LAUNCH(2, 248, true) COMBO_DIV_LAUNCH(2, 120, true) COMBO_DIV_LAUNCH(2, 56, true)
+            COMBO_DIV_LAUNCH_W(4, 252) COMBO_DIV_LAUNCH_W(4, 124) COMBO_DIV_LAUNCH_W(4, 60)
+            COMBO_DIV_LAUNCH_W(2, 248) COMBO_DIV_LAUNCH_W(2, 120) COMBO_DIV_LAUNCH_W(2, 56)
 #undef COMBO_DIV_LAUNCH
+#undef COMBO_DIV_LAUNCH_P
+#undef COMBO_DIV_LAUNCH_W
             if (e == cudaSuccess) e = cudaGetLastError();
             if (e != cudaSuccess) return cuda_fail(e, "divergence launch");
             t_last_path = 2;

@@ -21,6 +21,7 @@ constexpr int kDivSlots = 16;                          // rows a consumer warp c
 constexpr int kDivMaxStagedN = kDivSlots * kConsumerWarps;
 constexpr int kDivBox = 256;                           // widest TMA box in columns
 constexpr int kDivTile = 1024;                         // widest tile in columns (four boxes)
+constexpr int kDivWordMeans = 256;                     // floats per copy of the column means in word mode
 
 struct DivParams {
     const unsigned char* models;
@@ -31,6 +32,16 @@ struct DivParams {
     int N, narr, m, stages, row_bytes;
     unsigned coef_off, rowoff_off, part_off, mean_off, stage_off, stage_bytes;
 };
+
+// N consecutive floats of shared memory as one access (N = 1 or 2)
+template <int N_> __device__ __forceinline__ void store_floats_w(float* q, const float (&v)[N_]) {
+    if constexpr (N_ == 2) *reinterpret_cast<float2*>(q) = make_float2(v[0], v[1]);
+    else q[0] = v[0];
+}
+template <int N_> __device__ __forceinline__ void load_floats_w(const float* q, float (&v)[N_]) {
+    if constexpr (N_ == 2) { const float2 t = *reinterpret_cast<const float2*>(q); v[0] = t.x; v[1] = t.y; }
+    else v[0] = q[0];
+}
 
 // TC = columns per tile.  Rows that are 16-byte aligned: 64 to 1024 (the widest whose stage
 // stays within 64 KB; tiles wider than 256 columns are staged as several boxes, which keeps
@@ -127,6 +138,139 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
 #pragma unroll
     for (int s = 0; s < kDivSlots; ++s) acc[s] = 0.0;
 
+    if constexpr (WORD) {
+        // Rows with differing 16-byte phases: warp per row in both phases.  Warp cw owns rows
+        // cw, cw + 16, ...; lane l takes the 4-byte words l, l + 32, ... of a row (conflict-free
+        // whatever the row's phase), i.e. the same columns in every row, so that its column
+        // sums and, later, its column means stay in registers while it walks over its rows.
+        // Where a row lies in a stage does not depend on the tile: those offsets are registers
+        // too.  What goes through shared memory per row and phase is the row itself.
+        // bfloat16 operands enter binary32 adds directly (add.rn.f32.bf16: exact widening, one
+        // rounding); with unit weights the column sum needs no multiplication at all.
+        // The warp's rows are walked from the last to the first by a switch that falls through
+        // (straight-line code with fixed registers and no test per row).  A lane's last word
+        // may lie beyond the row's payload: it is read all the same (the bytes are inside the
+        // stage or its 16 bytes of slack); its column sums land in entries nobody reads, and
+        // for the deviations the word and its means are replaced by zero.
+        constexpr int WPL = (NU + 31) / 32;             // words per lane per row
+        constexpr int FPL = WPL * EPU;                  // binary32 values per lane per row
+        static_assert(NBX == 1, "word mode uses one box per tile");
+        int ro[kDivSlots];
+#pragma unroll
+        for (int sl = 0; sl < kDivSlots; ++sl) {
+            const int r = cw + sl * kConsumerWarps;
+            ro[sl] = r < N ? rowoff[r] : 0;
+        }
+        const int nrows = cw < N ? (N - cw + kConsumerWarps - 1) / kConsumerWarps : 0;
+        const bool weighted = p.weights != nullptr;
+        const float mscale = weighted ? 1.0f : coef[0];                 // unit weights: 1 / N
+        const bool tail_on = lane + 32 * (WPL - 1) < NU;               // the lane's last word exists
+        float* part_w = part + cw * (NUP * EPU);                       // this warp's column sums
+        const uint32_t lane_off = (uint32_t)lane * 4u;
+        const long long n_mine = (p.n_tiles > (long long)blockIdx.x)
+                                     ? (p.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+#define COMBO_DIV_CASES(ROW)                                                                             \
+    case 16: ROW(15) case 15: ROW(14) case 14: ROW(13) case 13: ROW(12) case 12: ROW(11) case 11: ROW(10) \
+    case 10: ROW(9) case 9: ROW(8) case 8: ROW(7) case 7: ROW(6) case 6: ROW(5) case 5: ROW(4)           \
+    case 4: ROW(3) case 3: ROW(2) case 2: ROW(1) case 1: ROW(0) default: break;
+        // One consumer-wide barrier per tile, as in vector mode (PIPE; needs three stages):
+        // step i sums tile i, and after the barrier forms its means and takes the deviations
+        // of tile i - 1 (two copies of the sums and of the means keep neighbouring steps apart).
+        for (long long i = 0; i <= n_mine; ++i) {
+            if (i < n_mine) {
+                const int s = (int)(i % stages);
+                if (!mbar_wait(smem_u32(&hdr->full[s]), (uint32_t)((i / stages) & 1))) { staged_fail(13); return; }
+                const uint32_t src_s = smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) +
+                                       (uint32_t)((p.narr - 1) * block_bytes) + lane_off;
+                // (A) column sums over this warp's rows
+                float a[FPL];
+#pragma unroll
+                for (int e = 0; e < FPL; ++e) a[e] = 0.0f;
+#define COMBO_DIV_ROW_A(SL)                                                                              \
+    {                                                                                                    \
+        const uint32_t row = src_s + (uint32_t)ro[SL];                                                   \
+        const float c = weighted ? coef[cw + SL * kConsumerWarps] : 1.0f;                                \
+        _Pragma("unroll") for (int q = 0; q < WPL; ++q) {                                                \
+            const uint32_t w = lds32<0>(row + 128u * q);                                                 \
+            if constexpr (EB == 4) {                                                                     \
+                a[q] = weighted ? fmaf(c, __uint_as_float(w), a[q]) : __fadd_rn(__uint_as_float(w), a[q]); \
+            } else if (weighted) {                                                                       \
+                a[2 * q] = fmaf(c, __uint_as_float(w << 16), a[2 * q]);                                  \
+                a[2 * q + 1] = fmaf(c, __uint_as_float(w & 0xffff0000u), a[2 * q + 1]);                  \
+            } else {                                                                                     \
+                a[2 * q] = add_bf16_lo(w, a[2 * q]);                                                     \
+                a[2 * q + 1] = add_bf16_hi(w, a[2 * q + 1]);                                             \
+            }                                                                                            \
+        }                                                                                                \
+    }
+                switch (nrows) { COMBO_DIV_CASES(COMBO_DIV_ROW_A) }
+#undef COMBO_DIV_ROW_A
+                float* pw = part_w + (i & 1) * (kConsumerWarps * NUP * EPU);
+#pragma unroll
+                for (int q = 0; q < WPL; ++q) {
+                    float v[EPU];
+#pragma unroll
+                    for (int e = 0; e < EPU; ++e) v[e] = a[q * EPU + e];
+                    store_floats_w<EPU>(pw + (lane + 32 * q) * EPU, v);
+                }
+            }
+            if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(14); return; }
+            if (i < n_mine) {
+                // (A2) column means: the warps' sums added in warp order
+                const float* pt = part + (i & 1) * (kConsumerWarps * NUP * EPU);
+                for (int c = ctid; c < TC; c += kConsumerThreads) {
+                    float m = 0.0f;
+#pragma unroll
+                    for (int g = 0; g < kConsumerWarps; ++g) m = __fadd_rn(m, pt[g * (NUP * EPU) + c]);
+                    mean[(i & 1) * kDivWordMeans + c] = __fmul_rn(m, mscale);
+                }
+            }
+            if (!PIPE) {
+                // too few stages to hold two tiles at a time: the deviations of tile i follow
+                // its means in the same step, behind a second barrier
+                if (!consumers_sync(csync, csync_phase, lane)) { staged_fail(15); return; }
+            }
+            if (PIPE ? (i >= 1) : (i < n_mine)) {
+                // (B) squared deviations of this warp's rows of tile t from the means of the
+                // lane's columns (pipelined: written in step i - 1, before this step's barrier)
+                const long long t = PIPE ? i - 1 : i;
+                const int s = (int)(t % stages);
+                const float* mn = mean + (t & 1) * kDivWordMeans;
+                float nmu[FPL];
+#pragma unroll
+                for (int q = 0; q < WPL; ++q) {
+                    float v[EPU];
+                    load_floats_w<EPU>(mn + (lane + 32 * q) * EPU, v);
+#pragma unroll
+                    for (int e = 0; e < EPU; ++e) nmu[q * EPU + e] = (q < WPL - 1 || tail_on) ? -v[e] : 0.0f;
+                }
+                const uint32_t own_s = smem_u32(smem + p.stage_off + (size_t)s * p.stage_bytes) + lane_off;
+#define COMBO_DIV_ROW_B(SL)                                                                              \
+    {                                                                                                    \
+        const uint32_t row = own_s + (uint32_t)ro[SL];                                                   \
+        float ssum = 0.0f;                                                                               \
+        _Pragma("unroll") for (int q = 0; q < WPL; ++q) {                                                \
+            uint32_t w = lds32<0>(row + 128u * q);                                                       \
+            if (q == WPL - 1) w = tail_on ? w : 0u;                                                      \
+            if constexpr (EB == 4) {                                                                     \
+                const float d = __fadd_rn(__uint_as_float(w), nmu[q]);                                   \
+                ssum = fmaf(d, d, ssum);                                                                 \
+            } else {                                                                                     \
+                const float d0 = add_bf16_lo(w, nmu[2 * q]), d1 = add_bf16_hi(w, nmu[2 * q + 1]);        \
+                ssum = fmaf(d0, d0, ssum);                                                               \
+                ssum = fmaf(d1, d1, ssum);                                                               \
+            }                                                                                            \
+        }                                                                                                \
+        acc[SL] += (double)ssum;                                                                         \
+    }
+                switch (nrows) { COMBO_DIV_CASES(COMBO_DIV_ROW_B) }
+#undef COMBO_DIV_ROW_B
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
+            }
+        }
+#undef COMBO_DIV_CASES
+    } else {
     // byte offset of unit u of a row inside an array's part of a stage (its box, then its place)
     auto unit_off = [&](int u) { return NBX == 1 ? u * UB : (u / UPB) * block_bytes + (u % UPB) * UB; };
     // one unit of a staged row as EPU binary32 values
@@ -243,6 +387,7 @@ k_divergence_staged(const DivParams p, const __grid_constant__ TileMaps maps) {
             if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
         }
     }
+    }   // vector mode
     // per-CTA partial sums: one entry per row, written by the warp that owns the row
 #pragma unroll
     for (int sl = 0; sl < kDivSlots; ++sl) {
