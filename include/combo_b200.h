@@ -33,7 +33,7 @@
  *               segment l; each (w,l) row ascending, all entries != w, distinct
  *   weights     float [N], |D_j| > 0, un-normalised; NULL = all equal
  *
- * Segments (Eq. 1; the paper's "divided into S segments equally"): segment
+ * Segments (Eq. 1; Section 5.1 cuts the model into S equal parts): segment
  * length L = ceil(P/S); segment l covers columns [min(l*L,P), min((l+1)*L,P)),
  * so the last segment is shorter when S does not divide P and trailing
  * segments may be empty.
@@ -189,8 +189,8 @@ combo_status combo_check_rows(const void* const* d_rows, int N, void* stream, in
 /*
  * Dynamic workers -- Section 4.2.
  *
- * combo_select_peers_online: a worker that is offline is not pulled from (the
- * requester "resends the request to another worker"), so every online worker
+ * combo_select_peers_online: a worker that is offline is not pulled from (its
+ * requester turns to some other worker instead), so every online worker
  * draws its peers from the ONLINE others only, by the same procedure as
  * combo_select_peers (identical tables when all are online).  An offline worker
  * issues no requests: its rows are filled with -1.  h_online: HOST array of N

@@ -379,10 +379,10 @@ int oracle_select_peers_active(uint64_t seed, uint32_t round, int N, int S, int 
 /* ------------------------------------------------------------------ */
 /* (2) Eq. 3 with the provider sets Section 4.2 allows:                */
 /*     P_l(w) = ({w} unless w is a newcomer) U {idx[w][l][r] >= 0}.    */
-/*     A new worker "pulls the segments and aggregates them as normal  */
-/*     only without its local model"; a negative idx entry is a pull   */
-/*     that found no online peer.  An empty P_l leaves the worker's    */
-/*     own values (reading: nothing to aggregate).                     */
+/*     A newcomer has no model of its own yet, so its aggregate is     */
+/*     formed from the pulled segments alone; a negative idx entry is  */
+/*     a pull that found no online peer.  An empty P_l leaves the      */
+/*     worker's own values (reading: nothing to aggregate).            */
 /*     newcomer: N bytes or NULL.  mode 0: binary64, quotient of sums, */
 /*     out = double; mode 1: the fixed-order binary32 form, out =      */
 /*     float (elem 4) or bf16 bits (elem 2).                           */

@@ -81,7 +81,7 @@ def test_both_kernels_agree_and_paths_are_taken():
 
 
 def test_round_with_all_replicas_has_no_divergence():
-    # R = n-1: "the model divergence decreases to zero" (Section 4.3); fewer replicas leave more
+    # R = n-1 leaves no divergence at all (Section 4.3); fewer replicas leave more
     N, P, S = 12, 120_000, 6
     x, _, w = make(N, P, torch.float32, 9)
     means = []

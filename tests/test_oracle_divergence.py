@@ -72,8 +72,8 @@ def test_translation_and_scaling_laws():
 
 
 def test_full_replica_round_has_zero_divergence_and_more_replicas_shrink_it():
-    # "If we let R = n-1 ... the model divergence decreases to zero" (Section 4.3), and the
-    # divergence "can be ameliorated by aggregating more models"
+    # Section 4.3: with R = n-1 no divergence is left, and pulling more replicas per segment
+    # shrinks it
     rng = np.random.default_rng(3)
     N, P, S = 10, 400, 5
     x = rng.normal(0, 0.05, (N, P)).astype(np.float32)
