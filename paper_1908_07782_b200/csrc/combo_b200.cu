@@ -929,9 +929,10 @@ combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, 
         q.ptr_off = 0;
         q.slot_off = round_up((unsigned)N * 8u, 128);
         q.list_off = q.slot_off + round_up((unsigned)N * 2u, 128);
-        q.tab_off = q.list_off + round_up((unsigned)d_max * 2u, 128);
+        q.tab_off = q.list_off + round_up((unsigned)d_max * 8u, 128);
         q.stage_off = q.tab_off + round_up(2u * (unsigned)n_local * (unsigned)combo::table_entry_bytes(rmax), 128);
         int T = 0;
+        // (the per-warp aggregation walks boxes of at most 256 columns, so tiles are no wider)
         for (int t = 256; t >= (elem_bytes == 4 ? 128 : 256); t >>= 1) {
             const long long need = (long long)q.stage_off + 3LL * d_max * t * elem_bytes + 16;
             if (need <= dev->smem_optin && t <= L) { T = t; break; }
@@ -949,6 +950,7 @@ combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, 
             q.n_local = n_local;
             q.T = T;
             q.row_bytes = T * elem_bytes;
+            for (q.gpr_log2 = 0; (16 << q.gpr_log2) < q.row_bytes; ++q.gpr_log2) {}
             q.d_max = (int)d_max;
             q.stage_bytes = (unsigned)(d_max * T * elem_bytes);
             q.n_tiles = (P + T - 1) / T;
@@ -963,16 +965,20 @@ combo_status combo_segment_aggregate_rows(const void* const* d_rows, void* out, 
             const size_t smem = (size_t)q.stage_off + (size_t)stages * (size_t)q.stage_bytes + 16;
             const int grid = (int)(q.n_tiles < dev->sms ? q.n_tiles : dev->sms);
             cudaError_t e = cudaErrorInvalidValue;
-#define COMBO_PULL_LAUNCH(EBV, RTV)                                                                              \
-    if (elem_bytes == EBV && rt == RTV) {                                                                        \
-        e = cudaFuncSetAttribute(combo::k_pull_staged<EBV, RTV>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
-                                 (int)smem);                                                                     \
-        if (e == cudaSuccess) combo::k_pull_staged<EBV, RTV><<<grid, combo::kPullThreads, smem, st>>>(q);        \
+            // bfloat16 rows with unit weights are summed by the mixed-precision add
+            const bool unw = elem_bytes == 2 && !weights;
+#define COMBO_PULL_LAUNCH(EBV, RTV, UNWV)                                                                        \
+    if (elem_bytes == EBV && rt == RTV && unw == UNWV) {                                                         \
+        e = cudaFuncSetAttribute(combo::k_pull_staged<EBV, RTV, UNWV>,                                           \
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);                        \
+        if (e == cudaSuccess) combo::k_pull_staged<EBV, RTV, UNWV><<<grid, combo::kPullThreads, smem, st>>>(q);  \
     }
-            COMBO_PULL_LAUNCH(4, 1) COMBO_PULL_LAUNCH(4, 2) COMBO_PULL_LAUNCH(4, 3) COMBO_PULL_LAUNCH(4, 4)
-            COMBO_PULL_LAUNCH(4, 8) COMBO_PULL_LAUNCH(4, -1) COMBO_PULL_LAUNCH(4, -2)
-            COMBO_PULL_LAUNCH(2, 1) COMBO_PULL_LAUNCH(2, 2) COMBO_PULL_LAUNCH(2, 3) COMBO_PULL_LAUNCH(2, 4)
-            COMBO_PULL_LAUNCH(2, 8) COMBO_PULL_LAUNCH(2, -1) COMBO_PULL_LAUNCH(2, -2)
+#define COMBO_PULL_LAUNCH_R(EBV, UNWV)                                                                           \
+    COMBO_PULL_LAUNCH(EBV, 1, UNWV) COMBO_PULL_LAUNCH(EBV, 2, UNWV) COMBO_PULL_LAUNCH(EBV, 3, UNWV)              \
+    COMBO_PULL_LAUNCH(EBV, 4, UNWV) COMBO_PULL_LAUNCH(EBV, 8, UNWV) COMBO_PULL_LAUNCH(EBV, -1, UNWV)             \
+    COMBO_PULL_LAUNCH(EBV, -2, UNWV)
+            COMBO_PULL_LAUNCH_R(4, false) COMBO_PULL_LAUNCH_R(2, false) COMBO_PULL_LAUNCH_R(2, true)
+#undef COMBO_PULL_LAUNCH_R
 #undef COMBO_PULL_LAUNCH
             if (e == cudaSuccess) e = cudaGetLastError();
             if (e != cudaSuccess) return cuda_fail(e, "staged pull aggregation launch");

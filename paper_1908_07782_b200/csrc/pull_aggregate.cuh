@@ -115,7 +115,8 @@ struct PullStagedParams {
     long long P, L, out_pitch, n_tiles;
     int N, S, R, w_begin, n_local;
     int T;                 // tile width in elements
-    int row_bytes;         // T * elem_bytes
+    int row_bytes;         // T * elem_bytes, a power of two
+    int gpr_log2;          // log2 of the 16-byte groups per staged row (row_bytes / 16 <= kPullThreads)
     int d_max;             // rows a stage has room for
     int stages;            // 3..8 stages of stage_bytes each
     unsigned ptr_off, slot_off, list_off, tab_off, stage_off, stage_bytes;
@@ -151,19 +152,19 @@ __device__ __forceinline__ void cp_async_wait_n(int n) {
 // in ascending worker order) and builds the coefficient table, whose provider offsets point
 // at those numbered slots of a stage.  Inside a run the tiles go through a ring of stages: the
 // loads of tile j + stages - 1 are issued before tile j is consumed, one copy group per tile.
-template <int EB, int RT>
+// UNW: bfloat16 rows with unit weights, summed by the mixed-precision add (see RowCtxU).
+template <int EB, int RT, bool UNW = false>
 __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStagedParams p) {
     constexpr int RMAX = (RT >= 0) ? RT : (RT == -2 ? kStagedMaxR : kGenericR);
-    constexpr int ENT = table_entry_bytes(RMAX);
+    constexpr int ENT = entry_bytes_of<RMAX, UNW>();
     extern __shared__ __align__(128) unsigned char smem[];
     const unsigned char** rowp = reinterpret_cast<const unsigned char**>(smem + p.ptr_off);
     short* slot_of = reinterpret_cast<short*>(smem + p.slot_off);     // [N]: stage slot of a worker's row or -1
-    short* need = reinterpret_cast<short*>(smem + p.list_off);        // [d_max]: worker of each slot
+    const unsigned char** srcp = reinterpret_cast<const unsigned char**>(smem + p.list_off);   // [d_max]: row held by each slot
     unsigned char* tab = smem + p.tab_off;                            // [2][n_local] entries
     __shared__ int s_nd;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = p.N, R = (RT >= 0) ? RT : p.R, nl = p.n_local;
-    const int groups_per_row = p.row_bytes / 16;
 
     for (int j = tid; j < N; j += kPullThreads) rowp[j] = static_cast<const unsigned char*>(p.rows[j]);
 
@@ -190,19 +191,20 @@ __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStage
     long long i = (long long)blockIdx.x * per;
     const long long i_end = i + per < p.n_tiles ? i + per : p.n_tiles;
 
+    // A thread copies the same 16-byte group of every sstep-th staged row (the groups per row
+    // are a power of two that divides the block size), so nothing is divided per copy.
+    const int my_g = tid & ((1 << p.gpr_log2) - 1), my_s0 = tid >> p.gpr_log2;
+    const int sstep = kPullThreads >> p.gpr_log2;
     auto issue = [&](long long tile, int st, int nd) {
         const long long t0 = tile * (long long)p.T;
-        const long long row_valid = (p.P - t0) * EB;                 // bytes of a row from t0 to its end
-        const uint32_t sbase = smem_u32(smem + p.stage_off + (size_t)st * p.stage_bytes);
-        const int total = nd * groups_per_row;
-        for (int q = tid; q < total; q += kPullThreads) {
-            const int s_ = q / groups_per_row, g = q - s_ * groups_per_row;
-            const long long left = row_valid - 16LL * g;
-            const int nb = left >= 16 ? 16 : (left > 0 ? (int)left : 0);
-            // a group wholly past the row's end reads nothing (its address is not formed)
-            const unsigned char* src = rowp[need[s_]] + (nb > 0 ? (size_t)t0 * EB + 16u * g : 0);
-            cp_async_16(sbase + (uint32_t)(s_ * p.row_bytes + 16 * g), src, nb);
-        }
+        const long long left = (p.P - t0) * EB - 16LL * my_g;        // bytes of a row from this group to its end
+        const int nb = left >= 16 ? 16 : (left > 0 ? (int)left : 0);
+        // a group wholly past the row's end reads nothing (its address is not formed)
+        const size_t off = nb > 0 ? (size_t)t0 * EB + 16u * my_g : 0;
+        uint32_t dst = smem_u32(smem + p.stage_off + (size_t)st * p.stage_bytes) +
+                       (uint32_t)(my_s0 * p.row_bytes + 16 * my_g);
+        const uint32_t dstep = (uint32_t)(sstep * p.row_bytes);
+        for (int s_ = my_s0; s_ < nd; s_ += sstep, dst += dstep) cp_async_16(dst, srcp[s_] + off, nb);
         cp_async_commit();
     };
 
@@ -244,11 +246,11 @@ __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStage
                 const unsigned b = __ballot_sync(0xffffffffu, bit);
                 if (bit) {
                     const int sl = nd + __popc(b & ((1u << lane) - 1u));
-                    if (sl < p.d_max) { slot_of[v] = (short)sl; need[sl] = (short)v; }
+                    if (sl < p.d_max) { slot_of[v] = (short)sl; srcp[sl] = rowp[v]; }
                 }
                 nd += __popc(b);
             }
-            for (int wi = lane; wi < nl; wi += 32) { slot_of[p.w_begin + wi] = (short)wi; need[wi] = (short)(p.w_begin + wi); }
+            for (int wi = lane; wi < nl; wi += 32) { slot_of[p.w_begin + wi] = (short)wi; srcp[wi] = rowp[p.w_begin + wi]; }
             if (lane == 0) s_nd = nd;
         }
         __syncthreads();
@@ -259,7 +261,7 @@ __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStage
             const int w = p.w_begin + wi;
             const int32_t* peers = p.idx + ((size_t)w * p.S + (size_t)(l0 + sg)) * (size_t)R;
             float* cf = reinterpret_cast<float*>(tab + ((size_t)sg * nl + wi) * ENT);
-            int* po = reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
+            int* po = UNW ? reinterpret_cast<int*>(cf) : reinterpret_cast<int*>(cf + 2 * (RMAX + 1));
             int prov[RMAX + 1];
             int np = 0;
             prov[np++] = w;
@@ -269,12 +271,21 @@ __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStage
             }
             float den = p.weights ? p.weights[prov[0]] : 1.0f;
             for (int t = 1; t < np; ++t) den = __fadd_rn(den, p.weights ? p.weights[prov[t]] : 1.0f);
-            cf[entry_scale_word(RMAX)] = np == 1 ? 1.0f : __fdiv_rn(1.0f, den);
+            const float scale = np == 1 ? 1.0f : __fdiv_rn(1.0f, den);
+            if (UNW) {
+                cf[RMAX + 1] = scale;
+                po[RMAX + 2] = np;
+            } else {
+                cf[entry_scale_word(RMAX)] = scale;
+            }
             for (int r = 0; r < np; ++r) {
-                cf[2 * r] = cf[2 * r + 1] = (np == 1 || !p.weights) ? 1.0f : p.weights[prov[r]];
+                if (!UNW) cf[2 * r] = cf[2 * r + 1] = (np == 1 || !p.weights) ? 1.0f : p.weights[prov[r]];
                 po[r] = (int)slot_of[prov[r]] * p.row_bytes;
             }
-            for (int r = np; r <= RMAX; ++r) { cf[2 * r] = cf[2 * r + 1] = 0.0f; po[r] = po[0]; }
+            for (int r = np; r <= RMAX; ++r) {
+                if (!UNW) cf[2 * r] = cf[2 * r + 1] = 0.0f;
+                po[r] = po[0];
+            }
         }
         __syncthreads();
 
@@ -295,7 +306,7 @@ __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStage
             if (j + NS - 1 < run_end) issue(j + NS - 1, (int)((j - i + NS - 1) % NS), nd);
             else cp_async_commit();
             unsigned char* stage = smem + p.stage_off + (size_t)st * p.stage_bytes;
-            aggregate_tile<EB, 16, RT>(ap, ws, stage, smem_u32(stage), tab, j, straddle ? bnd : (long long)1 << 62, lane);
+            aggregate_tile<EB, 16, RT, UNW>(ap, ws, stage, smem_u32(stage), tab, j, straddle ? bnd : (long long)1 << 62, lane);
         }
         cp_async_wait<0>();
         i = run_end;

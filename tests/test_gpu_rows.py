@@ -36,6 +36,11 @@ def make_rows(N, P, dtype, seed):
     (128, 30_008, 16, 4, 4, torch.bfloat16, True),
     (30, 100_000, 10, 12, 3, torch.float32, True),    # the wide kernel (R > 8)
     (12, 70_000, 5, 6, 2, torch.float32, False),      # the unspecialised one
+    # bfloat16 with unit weights: the mixed-precision sum, in each kernel instance
+    (128, 30_010, 16, 4, 4, torch.bfloat16, False),
+    (10, 9_999, 3, 1, 2, torch.bfloat16, False),
+    (20, 40_003, 6, 6, 2, torch.bfloat16, False),
+    (30, 60_000, 10, 12, 3, torch.bfloat16, False),
 ])
 @pytest.mark.parametrize("path", [0, 3])
 def test_rows_kernel_matches_oracle_and_dense_kernel(N, P, S, R, world, dtype, weighted, path):
@@ -80,14 +85,15 @@ def test_rows_kernel_matches_oracle_and_dense_kernel(N, P, S, R, world, dtype, w
     combo.combo_device_status()
 
 
+@pytest.mark.parametrize("weighted", [True, False])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-def test_rows_kernel_skips_pulls_that_found_no_peer(dtype):
+def test_rows_kernel_skips_pulls_that_found_no_peer(dtype, weighted):
     # a table from the online sampler holds -1 rows for offline workers and -1 pulls
     # (Section 4.2); the worker-sharded call must skip them like the dense kernels do
     N, P, S, R = 10, 20_003, 4, 3
     e = 4 if dtype == torch.float32 else 2
     dense, rows, table = make_rows(N, P, dtype, seed=5)
-    w = torch.randint(500, 1501, (N,), generator=torch.Generator().manual_seed(3)).float().to(DEV)
+    w = torch.randint(500, 1501, (N,), generator=torch.Generator().manual_seed(3)).float().to(DEV) if weighted else None
     active = np.ones(N, np.uint8)
     active[[2, 7]] = 0
     idx_np = oracle.select_peers_active(4, 1, N, S, R, active)
@@ -101,8 +107,8 @@ def test_rows_kernel_skips_pulls_that_found_no_peer(dtype):
     combo.combo_segment_aggregate_rows(table, out, pitch, e, w, idx, N, P, S, R, 0, N)
     torch.cuda.synchronize()
     got = out[:, :P].contiguous()
-    want = oracle.segment_aggregate_members(to_bits(dense), idx_np, S, R, w.cpu().numpy(), np.zeros(N, np.uint8),
-                                            ordered=True)
+    want = oracle.segment_aggregate_members(to_bits(dense), idx_np, S, R, w.cpu().numpy() if weighted else None,
+                                            np.zeros(N, np.uint8), ordered=True)
     assert (to_bits(got).view(np.uint8) == want.view(np.uint8)).all()
     # offline workers keep their values
     assert torch.equal(got[2], dense[2]) and torch.equal(got[7], dense[7])
