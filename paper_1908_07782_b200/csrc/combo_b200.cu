@@ -389,11 +389,12 @@ StagedPlan plan_tile(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, cons
     const unsigned header = round_up((unsigned)sizeof(combo::StagedHeader), 128);
     const unsigned table = round_up(2u * p.N * (unsigned)combo::table_entry_bytes(rmax), 128);
     // Tile: at least 1 KB of every row (256 binary32 or 512 bfloat16 columns; shorter row
-    // pieces cost HBM efficiency) and at least 8 KB in all, else as small as possible: the
+    // pieces cost HBM efficiency) and as close to 16 KB in all as it gets from below: the
     // smaller the tile, the more CTAs share an SM and the finer the hand-over between
-    // consecutive launches (measured on 2 to 32 rows of 1 M to 4 M elements: 8 rows of 1 M
-    // floats take 12.7 us with 8 KB tiles, 13.3 with 16 KB, 14.6 with 32 KB; tiles of 4 KB
-    // and less are far slower).  t_tile overrides.
+    // consecutive launches, but every tile pays its set-up once (measured: 8 rows of 1 M
+    // floats take 13.1 us with 8 KB tiles, 12.5 with 16 KB, 13.5 with 24 KB; 4 rows of 4 M
+    // 36.8 / 25.1 / 24.6 us with 4 / 8 / 12 KB; 2 rows of 4 M 29.4 / 17.4 / 14.1 us with
+    // 2 / 4 / 6 KB; 16 rows of 1 M 23.6 / 24.6 us with 16 / 32 KB).  t_tile overrides.
     int nbx = 0;
     for (int n = 1; n <= combo::kMaxBoxes; ++n) {
         if (256LL * n > p.L || narr * n > 32) break;
@@ -401,8 +402,9 @@ StagedPlan plan_tile(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, cons
             if (256 * n == t_tile) nbx = n;
             continue;
         }
+        // the widest tile of at most 16 KB, but never less than 1 KB of a row
+        if (nbx > 0 && 256 * nbx * EB >= 1024 && (long long)narr * n * p.N * 256 * EB > 16 * 1024) break;
         nbx = n;
-        if (256 * n * EB >= 1024 && (long long)narr * n * p.N * 256 * EB >= 8 * 1024) break;
     }
     if (nbx == 0) return plan;
     const long long stage = (long long)narr * nbx * p.N * 256 * EB;
