@@ -169,9 +169,11 @@ combo_status combo_segment_aggregate_cols(const void* params_in, const void* gra
  * models of the n_local workers w_begin .. w_begin + n_local - 1 that this
  * GPU hosts and writes them to out, [n_local][out_pitch] (out_pitch >= P
  * elements, out_pitch * elem_bytes a multiple of 16; must not overlap any
- * row).  A pull is a plain load of W_k[l] from where worker k lives: per
- * hosted worker exactly R segments per segment index cross to this GPU, as in
- * the paper.  idx is the full [N][S][R] table (every GPU computes the same
+ * row).  A pull is a plain load of W_k[l] from where worker k lives (no bulk
+ * copy, no multicast); a segment of a peer that several hosted workers pull
+ * is loaded once per column tile and shared, so per segment index at most R
+ * segments per hosted worker cross to this GPU -- the paper's count, less the
+ * shared ones.  idx is the full [N][S][R] table (every GPU computes the same
  * one from the seed), weights the full [N] array or NULL.  Same arithmetic and
  * order as combo_segment_aggregate.  The caller orders the rounds: rows must
  * be final before the call (Section 4.1: a worker sends after its local

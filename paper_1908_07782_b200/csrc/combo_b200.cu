@@ -430,11 +430,12 @@ StagedPlan plan_tile(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, cons
     plan.ok = plan.grid > 0;
     (void)V;
     // Taken automatically where it measured faster than the persistent kernel's ring: tiles of
-    // 8 to 16 KB (up to 16 rows), which let a dozen or more CTAs share an SM, and at most two
-    // replicas.  (8 x 1 M floats, R = 2: 12.8 us against 13.6; 16 x 1 M: 23.2 against 24.4;
-    // 2 x 4 M, R = 1: 12.1 against 18.9.  With R = 3 or 4 the ring wins by 10 to 15 %, with 24
-    // and more rows it is as good or better, bfloat16 tiles of 8 KB lose 5 %.)
-    *short_enough = stage >= 8 * 1024 && stage <= 16 * 1024 && p.R <= 2 && (EB == 4 || stage == 16 * 1024) &&
+    // 8 to 24 KB (up to 24 rows), which let nine or more CTAs share an SM, and at most two
+    // replicas.  (8 x 1 M floats, R = 2: 12.5 us against 13.6; 16 x 1 M: 23.5 against 24.4;
+    // 24 x 1 M: 34.1 against 35.3; 2 x 64 M, R = 1: 163 against 260; 8 x 64 M: 635 against 638.
+    // With R = 3 or 4 the ring wins by 2 to 10 %, with 32 and more rows it is as good or
+    // better, bfloat16 tiles of 8 KB lose 5 %.)
+    *short_enough = stage >= 8 * 1024 && stage <= 24 * 1024 && p.R <= 2 && (EB == 4 || stage >= 16 * 1024) &&
                     p.n_tiles <= kTileMaxCtas;
     return plan;
 }
