@@ -248,11 +248,13 @@ StagedPlan plan_staged(AggParams& p, combo::TileMaps& maps, int EB, bool sgd, co
     }
     const Cand c = cands[pick];
     if (plan.rt == -3 && c.box_w != 256) plan.rt = -2;   // the dense form walks whole 512-byte chunks of 256-column boxes
-    // Measured on B200: throughput peaks with about 96-128 KB of loads in flight per SM and
-    // drops by 5-10 % beyond that, so the ring is kept that short (at least two stages; stages of
-    // at most 32 KB, which fill and drain more often, may hold up to 160 KB together).
+    // Measured on B200: throughput peaks with about 128-160 KB of staged data per SM (the stage
+    // being consumed included) and drops by up to 5-10 % beyond that on some GPUs, so the ring is
+    // kept that short: two stages of 64 KB, else as many as stay within 160 KB (48 rows of
+    // binary32, 48 KB stages: 0.93 with two, 0.97 with three; 40 rows: 0.89 / 0.97; a third
+    // stage of 64 KB gave +2 % to -1.6 % depending on shape and GPU).
     const int fit = (int)(budget / stage_bytes(c));
-    int stages = (int)(((stage_bytes(c) <= 32 * 1024 ? 160 : 112) * 1024) / stage_bytes(c));
+    int stages = (int)(((stage_bytes(c) < 64 * 1024 ? 160 : 128) * 1024) / stage_bytes(c));
     if (stages < 2) stages = 2;
     if (t_stages > 0) stages = t_stages;
     if (stages > combo::kMaxStages) stages = combo::kMaxStages;
