@@ -75,3 +75,31 @@ def test_random_long_rows(seed):
         check_against_oracle(x[:, c0:c1].contiguous(), a[:, c0:c1].contiguous(), idx_np, S, R, weights=w,
                              grads=grads[:, c0:c1].contiguous() if fused else None, lr=0.01, P=P, p_begin=c0)
     combo.combo_device_status()
+
+
+@pytest.mark.parametrize("N,P,S,R,dtype,weighted", [
+    (40, 1_300_004, 10, 4, torch.float32, False),     # 40 KB stages: a ring of four
+    (48, 1_250_000, 7, 3, torch.float32, True),       # 48 KB stages: a ring of three
+    (80, 1_300_008, 16, 4, torch.bfloat16, False),    # aligned bf16 rows, 40 KB stages
+    (100, 1_300_002, 16, 4, torch.bfloat16, True),    # rows of differing phase, 50 KB stages
+    (20, 1_300_000, 5, 2, torch.float32, False),      # with gradients beside the parameters: 40 KB stages
+])
+def test_long_kernels_with_deeper_rings(N, P, S, R, dtype, weighted):
+    # many rows and tens of tiles per CTA: stages below 64 KB, of which the ring holds three or
+    # four; whole-array equality with the direct kernel, windows against the oracle
+    fused = dtype == torch.float32 and N == 20
+    g = torch.Generator().manual_seed(N)
+    x = (torch.randn(N, P, generator=g) * 0.05).to(dtype).to(DEV)
+    grads = (torch.randn(N, P, generator=g) * 1e-3).to(DEV) if fused else None
+    w = torch.randint(500, 1501, (N,), generator=g).float().to(DEV) if weighted else None
+    idx_np = oracle.select_peers(N, 2, N, S, R)
+    idx = torch.from_numpy(idx_np).to(DEV)
+    a, used = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01)
+    assert used == combo.PATH_STAGED
+    b, _ = gpu_aggregate(x, idx, S, R, weights=w, grads=grads, lr=0.01, path=combo.PATH_DIRECT)
+    assert torch.equal(a, b), (N, P, S, R, dtype)
+    L = -(-P // S)
+    for (c0, c1) in ((0, 1500), (L - 700, L + 700), (P - 1500, P)):
+        check_against_oracle(x[:, c0:c1].contiguous(), a[:, c0:c1].contiguous(), idx_np, S, R, weights=w,
+                             grads=grads[:, c0:c1].contiguous() if fused else None, lr=0.01, P=P, p_begin=c0)
+    combo.combo_device_status()
