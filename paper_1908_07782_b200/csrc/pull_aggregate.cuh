@@ -114,9 +114,11 @@ struct PullStagedParams {
     const int32_t* idx;
     long long P, L, out_pitch, n_tiles;
     int N, S, R, w_begin, n_local;
-    int T;                 // tile width in elements
-    int row_bytes;         // T * elem_bytes, a power of two
-    int gpr_log2;          // log2 of the 16-byte groups per staged row (row_bytes / 16 <= kPullThreads)
+    int T;                 // tile width in elements: nbx boxes of row_bytes / elem_bytes columns
+    int nbx;               // x-boxes per tile, a power of two; a stage is [nbx][d_max][row_bytes]
+    int row_bytes;         // bytes of a staged row of one box, a power of two
+    int gpr_log2;          // log2 of the 16-byte groups of a row's tile piece (nbx * row_bytes / 16 <= kPullThreads)
+    int gpb_log2;          // log2 of the 16-byte groups per box row (row_bytes / 16)
     int d_max;             // rows a stage has room for
     int stages;            // 3..8 stages of stage_bytes each
     unsigned ptr_off, slot_off, list_off, tab_off, stage_off, stage_bytes;
@@ -181,9 +183,11 @@ __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStage
     ap.R = p.R;
     ap.T = p.T;
     ap.m = 1;
-    ap.nbx = 1;
-    ap.box_w = p.T;
+    ap.nbx = p.nbx;
+    ap.box_w = p.T / p.nbx;
     ap.row_bytes = p.row_bytes;
+    ap.stage_rows = p.d_max;
+    ap.dslot_bytes = 0;
     const WarpShare<EB, 16> ws(ap, warp, kPullWarps, lane);
 
     // contiguous share of the tiles
@@ -201,8 +205,10 @@ __global__ void __launch_bounds__(kPullThreads, 1) k_pull_staged(const PullStage
         const int nb = left >= 16 ? 16 : (left > 0 ? (int)left : 0);
         // a group wholly past the row's end reads nothing (its address is not formed)
         const size_t off = nb > 0 ? (size_t)t0 * EB + 16u * my_g : 0;
+        // group my_g of the tile piece lies in box my_g >> gpb_log2
         uint32_t dst = smem_u32(smem + p.stage_off + (size_t)st * p.stage_bytes) +
-                       (uint32_t)(my_s0 * p.row_bytes + 16 * my_g);
+                       (uint32_t)((my_g >> p.gpb_log2) * p.d_max * p.row_bytes + my_s0 * p.row_bytes +
+                                  16 * (my_g & ((1 << p.gpb_log2) - 1)));
         const uint32_t dstep = (uint32_t)(sstep * p.row_bytes);
         for (int s_ = my_s0; s_ < nd; s_ += sstep, dst += dstep) cp_async_16(dst, srcp[s_] + off, nb);
         cp_async_commit();

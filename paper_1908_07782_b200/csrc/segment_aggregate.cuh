@@ -98,6 +98,7 @@ struct AggParams {
     int tab_slots;       // segments the table holds: all S of them, or 2 (rebuilt on the way)
     unsigned dtab_off;   // byte offset of the dense coefficient blocks (dense mode only)
     int dslot_bytes;     // bytes of one segment's dense blocks
+    int stage_rows;      // rows between the x-boxes of a staged tile; 0 = N (a stage may have room for more rows than it holds)
     unsigned stage_off;  // byte offset of stage 0
     unsigned stage_bytes;
     TileSlot* sched;     // tile dispenser of this launch
@@ -1107,7 +1108,7 @@ __device__ __forceinline__ void aggregate_tile(const AggParams& p, const WarpSha
     constexpr int PSTRIDE = WarpShare<EB, GB>::PSTRIDE;
     constexpr int EPP = GB / EB;               // elements per piece
     const int N = p.N, R = (RT >= 0) ? RT : p.R;
-    const int block_bytes = N * p.row_bytes;               // one x-box of all rows
+    const int block_bytes = (p.stage_rows ? p.stage_rows : N) * p.row_bytes;   // one x-box of all rows
     const int box_payload = ws.box_payload;
     const size_t pitch_bytes = ws.pitch_bytes;
     const int u_begin = ws.u_begin, u_end = ws.u_end;

@@ -36,6 +36,13 @@ def make_rows(N, P, dtype, seed):
     (128, 30_008, 16, 4, 4, torch.bfloat16, True),
     (30, 100_000, 10, 12, 3, torch.float32, True),    # the wide kernel (R > 8)
     (12, 70_000, 5, 6, 2, torch.float32, False),      # the unspecialised one
+    # few hosted rows: tiles of several boxes (2, 4 and 8; bfloat16 up to 1024 columns)
+    (16, 300_004, 5, 3, 1, torch.float32, True),
+    (16, 300_004, 5, 3, 4, torch.float32, False),     # 4 hosted workers
+    (6, 200_001, 3, 2, 1, torch.float32, False),      # 6 rows: 1024 columns per tile, ragged end
+    (3, 150_000, 2, 1, 3, torch.float32, True),       # one hosted worker: 2048 columns
+    (24, 260_010, 7, 4, 2, torch.bfloat16, False),
+    (24, 260_010, 7, 4, 1, torch.bfloat16, True),
     # bfloat16 with unit weights: the mixed-precision sum, in each kernel instance
     (128, 30_010, 16, 4, 4, torch.bfloat16, False),
     (10, 9_999, 3, 1, 2, torch.bfloat16, False),
