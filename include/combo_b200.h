@@ -330,7 +330,9 @@ void combo_set_kernel_path(int path);
  * (a multiple of 256 up to 2048; for rows whose byte pitch is not a multiple
  * of 16 every 256 asked for become 256 - 16/elem_bytes) and number of pipeline
  * stages; 0 = chosen automatically.  A tile that cannot be honoured makes
- * the call fall back to the direct kernel. */
+ * the call fall back to the direct kernel.  combo_segment_aggregate_rows takes
+ * the widest 256 * 2^k columns that do not exceed the tile asked for, and at
+ * least three stages. */
 void combo_set_tuning(int tile_elems, int stages);
 
 /* This thread only: whether the staged aggregation kernel is launched with
